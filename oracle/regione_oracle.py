@@ -1,0 +1,388 @@
+"""fp64 CPU oracle for the region-aware denoising step (RegionE, arXiv 2510.25590).
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product path may import this file;
+only tests, the smoke check and the benchmark's CPU-baseline leg use it.  It
+shares no code with the CUDA path and imports nothing from it.
+
+Every function is the plain definition the paper gives, evaluated in float64
+with numpy, without blocking, fusion or reordering.  Inputs are arrays whose
+values are already bf16-representable (the caller widens them); outputs stay
+float64.  Index outputs are int32.
+
+Pins (see tests, marker "not gpu"): straight-line identity, Euler invariance,
+planted-mask recovery, index invariants, scatter(gather) round trip, plain
+copy for the identity keep list, brute-force loops on tiny shapes, agreement
+with a library softmax-attention, split/permutation invariance, uniform-key
+mean, dominant-key selection, the gamma = 1 closed form of the appendix, and
+the zero-edit / full-edit merge cases.  No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+COSINE = 0
+L2 = 1
+
+
+def _f64(a):
+    return np.asarray(a, dtype=np.float64)
+
+
+# ----------------------------------------------------------------------------
+# Adaptive Region Partition
+# ----------------------------------------------------------------------------
+
+
+def one_step_estimate(x_t, t, v):
+    """One-step clean estimate: X_hat_0 = X_t - v * (t - 0).
+
+    One-step estimation equation of the Adaptive Region Partition paragraph
+    with t_f = 0; Algorithm 1, the line computing X_hat_0.
+    """
+    return _f64(x_t) - float(t) * _f64(v)
+
+
+def token_score(x0_hat, ref, metric):
+    """One score per token, reduced over that token's channels.
+
+    metric COSINE: cosine similarity between the estimate and the instruction
+    (reference) latent "along the token dimension" (Adaptive Region Partition
+    paragraph).  A zero denominator is clamped at 1e-12.
+    metric L2: Euclidean distance over the channels (not squared, not averaged).
+    """
+    a, r = _f64(x0_hat), _f64(ref)
+    if metric == COSINE:
+        dot = np.sum(a * r, axis=-1)
+        den = np.sqrt(np.sum(a * a, axis=-1)) * np.sqrt(np.sum(r * r, axis=-1))
+        return dot / np.maximum(den, 1e-12)
+    if metric == L2:
+        d = a - r
+        return np.sqrt(np.sum(d * d, axis=-1))
+    raise ValueError("metric")
+
+
+def edit_mask(score, metric, threshold):
+    """mask = 1 (edited) unless the token is "sufficiently similar" to the reference.
+
+    Cosine: the paper calls a token unedited iff similarity > eta (strict), so
+    it is edited iff s <= eta.  L2: edited iff distance > tau, unedited iff
+    distance <= tau.
+    """
+    s = _f64(score)
+    thr = float(threshold)
+    if metric == COSINE:
+        return (s <= thr).astype(np.uint8)
+    if metric == L2:
+        return (s > thr).astype(np.uint8)
+    raise ValueError("metric")
+
+
+def compact_indices(mask):
+    """E_index, U_index (ascending token ids), slot and count for one request.
+
+    Algorithm 1: E_index / U_index used by X[E_index], X[U_index].  A plain
+    sequential loop; ``slot[n]`` is the position of token n in ``edit_idx`` or -1.
+    Entries of edit_idx past n_edit and of keep_idx past N - n_edit are -1 here
+    (the GPU leaves them untouched; tests compare the live prefix only).
+    """
+    m = np.asarray(mask).astype(bool)
+    N = m.shape[0]
+    edit_idx = np.full(N, -1, np.int32)
+    keep_idx = np.full(N, -1, np.int32)
+    slot = np.full(N, -1, np.int32)
+    ne = 0
+    nk = 0
+    for n in range(N):
+        if m[n]:
+            edit_idx[ne] = n
+            slot[n] = ne
+            ne += 1
+        else:
+            keep_idx[nk] = n
+            nk += 1
+    return edit_idx, keep_idx, slot, ne
+
+
+def partition(x_t, v, ref, t, metric, threshold):
+    """Adaptive Region Partition without the morphological clean-up.
+
+    x_t, v, ref: [B, N, C].  Returns dict(score [B,N] f64, mask u8 [B,N],
+    edit_idx, keep_idx, slot int32 [B,N], n_edit int32 [B]).
+    """
+    x_t, v, ref = _f64(x_t), _f64(v), _f64(ref)
+    B, N, _ = x_t.shape
+    score = token_score(one_step_estimate(x_t, t, v), ref, metric)
+    mask = edit_mask(score, metric, threshold)
+    edit_idx = np.empty((B, N), np.int32)
+    keep_idx = np.empty((B, N), np.int32)
+    slot = np.empty((B, N), np.int32)
+    n_edit = np.empty(B, np.int32)
+    for b in range(B):
+        edit_idx[b], keep_idx[b], slot[b], n_edit[b] = compact_indices(mask[b])
+    return dict(score=score, mask=mask, edit_idx=edit_idx, keep_idx=keep_idx, slot=slot,
+                n_edit=n_edit)
+
+
+# ----------------------------------------------------------------------------
+# Morphological opening + closing of the edited mask (ARP clean-up step)
+# ----------------------------------------------------------------------------
+
+
+def _erode3(m):
+    """3x3 binary erosion; neighbours outside the grid are ignored."""
+    rows, cols = m.shape
+    out = np.ones_like(m)
+    for dr in (-1, 0, 1):
+        for dc in (-1, 0, 1):
+            for r in range(rows):
+                for c in range(cols):
+                    rr, cc = r + dr, c + dc
+                    if 0 <= rr < rows and 0 <= cc < cols and not m[rr, cc]:
+                        out[r, c] = 0
+    return out
+
+
+def _dilate3(m):
+    """3x3 binary dilation; neighbours outside the grid are ignored."""
+    rows, cols = m.shape
+    out = np.zeros_like(m)
+    for dr in (-1, 0, 1):
+        for dc in (-1, 0, 1):
+            for r in range(rows):
+                for c in range(cols):
+                    rr, cc = r + dr, c + dc
+                    if 0 <= rr < rows and 0 <= cc < cols and m[rr, cc]:
+                        out[r, c] = 1
+    return out
+
+
+def open_close(mask, grid):
+    """Opening (erode, dilate) then closing (dilate, erode) of the edited mask.
+
+    The Adaptive Region Partition paragraph applies "morphological opening and
+    closing"; the structuring element is not given: a 3x3 square on the
+    rows x cols token grid is used, out-of-grid neighbours ignored.
+    """
+    m = np.asarray(mask).astype(np.uint8).reshape(grid)
+    m = _dilate3(_erode3(m))
+    m = _erode3(_dilate3(m))
+    return m.reshape(-1)
+
+
+# ----------------------------------------------------------------------------
+# Token gather / scatter, RIKV cache store
+# ----------------------------------------------------------------------------
+
+
+def gather(src, idx, n):
+    """dst[b, j] = src[b, idx[b, j]] for j < n[b]  (X^E = X[E_index]; Algorithm 1).
+
+    Rows j >= n[b] of the result are NaN (unspecified on the GPU).
+    """
+    src = np.asarray(src)
+    idx = np.asarray(idx)
+    B = src.shape[0]
+    cap = idx.shape[1]
+    dst = np.full((B, cap) + src.shape[2:], np.nan, dtype=np.float64)
+    for b in range(B):
+        for j in range(int(n[b])):
+            dst[b, j] = src[b, idx[b, j]]
+    return dst
+
+
+def scatter(dst, src, idx, n):
+    """dst[b, idx[b, j]] = src[b, j] for j < n[b]; other rows of dst unchanged.
+
+    The re-gathering of region results by spatial position (end of the
+    Adaptive Velocity Decay Cache paragraph; Algorithm 1, the gather line).
+    """
+    out = np.array(dst, dtype=np.float64, copy=True)
+    for b in range(out.shape[0]):
+        for j in range(int(n[b])):
+            out[b, idx[b, j]] = src[b, j]
+    return out
+
+
+def rikv_store(k_full, v_full, keep_rows, n_keep):
+    """K^C, V^C: the retained rows of the last full step's K and V.
+
+    Stabilization Stage paragraph ("save the Key and Value in each attention
+    layer"), refreshed at forced steps.  k_full, v_full: [B, n_full, H, D];
+    keep_rows [B, cap]; returns (k_cache, v_cache) [B, cap, H, D], NaN past n_keep[b].
+    """
+    return gather(k_full, keep_rows, n_keep), gather(v_full, keep_rows, n_keep)
+
+
+# ----------------------------------------------------------------------------
+# Region attention with the Region-Instruction KV cache
+# ----------------------------------------------------------------------------
+
+
+def region_attention(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, scale=None):
+    """softmax(Q [K_fresh, K_cache]^T / sqrt(d)) [V_fresh, V_cache].
+
+    The attention equation of the Region-Aware Generation paragraph: queries of
+    the recomputed tokens against the concatenation of their own fresh keys
+    and the cached keys of everything else.  The concatenation is written out
+    literally.  q [B, Nq, H, D]; k/v fresh [B, Nf, H, D]; cache [B, Nc, H, D];
+    counts per batch entry.  Rows q >= n_q[b] of the result are NaN.  With no
+    key at all the result row is zero.
+    """
+    q = _f64(q)
+    B, Nq, H, D = q.shape
+    s = (1.0 / np.sqrt(D)) if scale is None or scale <= 0 else float(scale)
+    out = np.full((B, Nq, H, D), np.nan)
+    for b in range(B):
+        nq, nf, nc = int(n_q[b]), int(n_fresh[b]), int(n_cache[b])
+        if nq == 0:
+            continue
+        if nf + nc == 0:
+            out[b, :nq] = 0.0
+            continue
+        K = np.concatenate([_f64(k_fresh[b, :nf]), _f64(k_cache[b, :nc])], axis=0)
+        V = np.concatenate([_f64(v_fresh[b, :nf]), _f64(v_cache[b, :nc])], axis=0)
+        for h in range(H):
+            logits = (q[b, :nq, h, :] @ K[:, h, :].T) * s
+            logits = logits - logits.max(axis=1, keepdims=True)
+            p = np.exp(logits)
+            p = p / p.sum(axis=1, keepdims=True)
+            out[b, :nq, h, :] = p @ V[:, h, :]
+    return out
+
+
+def region_attention_rows(q, k_fresh, v_fresh, k_cache, v_cache, n_fresh, n_cache, samples,
+                          scale=None):
+    """Same definition, evaluated only at sampled (b, q_row, h) triples.
+
+    Returns [len(samples), D].  Used for parity at sizes where the full oracle
+    would take too long.
+    """
+    D = np.shape(q)[-1]
+    s = (1.0 / np.sqrt(D)) if scale is None or scale <= 0 else float(scale)
+    res = np.empty((len(samples), D))
+    for i, (b, r, h) in enumerate(samples):
+        nf, nc = int(n_fresh[b]), int(n_cache[b])
+        K = np.concatenate([_f64(k_fresh[b, :nf, h]), _f64(k_cache[b, :nc, h])], axis=0)
+        V = np.concatenate([_f64(v_fresh[b, :nf, h]), _f64(v_cache[b, :nc, h])], axis=0)
+        logits = (K @ _f64(q[b, r, h])) * s
+        logits = logits - logits.max()
+        p = np.exp(logits)
+        p = p / p.sum()
+        res[i] = p @ V
+    return res
+
+
+# ----------------------------------------------------------------------------
+# Adaptive Velocity Decay cache
+# ----------------------------------------------------------------------------
+
+
+def decay_factor(dt, gamma):
+    """(1 - dt) * gamma: the per-step decay of the velocity norm (decay-factor equation)."""
+    return (1.0 - float(dt)) * float(gamma)
+
+
+def avd_step(running_product, dt, gamma, delta):
+    """One step of the AVDCache criterion.
+
+    Criterion = 1 - prod (1 - dt) * gamma accumulated since the cached step
+    (criterion equation).  Returns (new_product, reuse).  If the criterion
+    exceeds delta the DiT is recomputed: the cache is refreshed and the product
+    restarts at 1.  Otherwise the cached velocity times the product is used.
+    """
+    p = float(running_product) * decay_factor(dt, gamma)
+    if 1.0 - p > float(delta):
+        return 1.0, False
+    return p, True
+
+
+def avd_schedule(timesteps, gammas, delta, first, last):
+    """Decisions for region steps j = first, first-1, ..., last (descending step index).
+
+    The first step of a run always computes (empty cache).  Returns a list of
+    (j, reuse, scale) with scale the factor applied to the cached velocity.
+    ``timesteps[i]`` = t_i, increasing in i; the step at index j advances from
+    t_j to t_{j-1}; its decay factor uses dt = t_{j+1} - t_j and gamma_{t_j}.
+    """
+    out = []
+    prod = 1.0
+    have_cache = False
+    for j in range(first, last - 1, -1):
+        if not have_cache:
+            out.append((j, False, 1.0))
+            have_cache = True
+            prod = 1.0
+            continue
+        prod, reuse = avd_step(prod, timesteps[j + 1] - timesteps[j], gammas[j], delta)
+        out.append((j, reuse, prod if reuse else 1.0))
+    return out
+
+
+def velocity_decay(v_in, scale, dt, x_e, n_edit):
+    """v^E = scale * v_in;  X^E_{t_{j-1}} = X^E_{t_j} - dt * v^E  (Euler sampler equation).
+
+    ``scale`` is the accumulated decay product when the cached velocity is
+    reused and 1 on a recomputed step.  Rows >= n_edit[b] are returned unchanged.
+    Returns (x_e_new, v_used).
+    """
+    v_in, x_e = _f64(v_in), _f64(x_e)
+    v_used = float(scale) * v_in
+    x_new = np.array(x_e, copy=True)
+    for b in range(x_e.shape[0]):
+        ne = int(n_edit[b])
+        x_new[b, :ne] = x_e[b, :ne] - float(dt) * v_used[b, :ne]
+    return x_new, v_used
+
+
+# ----------------------------------------------------------------------------
+# Merge of the two regions
+# ----------------------------------------------------------------------------
+
+
+def merge(x_full, v_last_full, x_e, slot, dt_unedited):
+    """Full image tokens after a run of region steps.
+
+    Edited tokens come from the iterated X^E (by slot); unedited tokens are the
+    one-step prediction X^U - v^U * dt with the last full step's velocity
+    (one-step estimation equation; Algorithm 1, the two lines before and after
+    the inner loop).
+    """
+    x_full, v_last_full, x_e = _f64(x_full), _f64(v_last_full), _f64(x_e)
+    B, N, _ = x_full.shape
+    out = np.empty_like(x_full)
+    for b in range(B):
+        for n in range(N):
+            j = int(slot[b, n])
+            if j >= 0:
+                out[b, n] = x_e[b, j]
+            else:
+                out[b, n] = x_full[b, n] - float(dt_unedited) * v_last_full[b, n]
+    return out
+
+
+# ----------------------------------------------------------------------------
+# Stage schedule (host control flow of Algorithm 1)
+# ----------------------------------------------------------------------------
+
+
+def stage_schedule(T=28, t_st=6, forced=(16,), t_sm=2):
+    """Step kinds for steps T, T-1, ..., 1.
+
+    Stabilization: steps T .. T-t_st+1 are full; the last of them stores K/V.
+    Bounds [T-t_st, *forced, t_sm-1].  For each consecutive (prev, next):
+    region steps prev .. next+2, a merge, then one full step at next+1 that
+    refreshes the cache.  Steps below the last bound are full smooth steps.
+    Returns a list of (step_index, kind) with kind in {"full", "full_store",
+    "region"}; a merge precedes every "full_store" that follows region steps.
+    """
+    kinds = []
+    for i in range(T, T - t_st, -1):
+        kinds.append((i, "full_store" if i == T - t_st + 1 else "full"))
+    bounds = [T - t_st] + list(forced) + [t_sm - 1]
+    for prev, nxt in zip(bounds[:-1], bounds[1:]):
+        for j in range(prev, nxt + 1, -1):
+            kinds.append((j, "region"))
+        kinds.append((nxt + 1, "full_store"))
+    for i in range(bounds[-1], 0, -1):
+        kinds.append((i, "full"))
+    return kinds
