@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the region-aware denoising step (RegionE hot path) on B200.
+
+A "step" is one pass of the whole hot path over one batch of synthetic input of
+the FLUX-Kontext-shaped workload (4096 image + 4096 reference + 512 text tokens,
+24 heads x 128, two-ellipse 20 % edit mask): partition, row lists, gathers, RIKV
+store, region attention, scatter, velocity decay + Euler, merge (12 launches).
+
+Prints ONE JSON line (rank 0).  `value` = region-attention FLOPs of the step
+divided by the whole step's device time (inputs resident in HBM).  `roofline`
+covers the dominant kernel (the attention) timed by CUDA events inside the
+same timed steps.  `--impl reference` times the fp64 CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "region-attention TFLOP/s over the whole region-aware denoise step"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                        bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                        source="measured")
+        except Exception:
+            pass
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def recorded_traffic():
+    """DRAM bytes per attention launch from the committed ncu summary, if any (else None)."""
+    path = os.path.join(ROOT, "profiles", "roofline_traffic.json")
+    if os.path.exists(path):
+        try:
+            return json.load(open(path)).get("region_attention_config2_dram_bytes_per_launch")
+        except Exception:
+            return None
+    return None
+
+
+def shard_requests(total: int, world_size: int, rank: int):
+    """Contiguous shard of `total` independent requests for `rank` (no data-path collective)."""
+    base, extra = divmod(total, world_size)
+    start = rank * base + min(rank, extra)
+    return list(range(start, start + base + (1 if rank < extra else 0)))
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nme, val in zip(names, parts[3:7]):
+                if val == "Active":
+                    reasons.add(nme)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def attention_flops(n_q, n_kv, H, D):
+    return float(4.0 * H * D * np.sum(n_q.astype(np.float64) * n_kv.astype(np.float64)))
+
+
+def make_workload(cfg: int, stream: int):
+    from paper_2510_25590_b200 import synth
+    wl = synth.WORKLOADS[cfg]
+    lat = synth.make_latents(wl, stream=stream)
+    qkv = synth.make_qkv_full(wl, stream=stream)
+    return wl, lat, qkv
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def time_oracle(wl, lat, qkv, heads, steps, warmup):
+    from oracle import step_oracle
+    t, scale, dt, dt_u = lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0
+    times = []
+    res = None
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        res = step_oracle.region_step(wl, lat, qkv, t, scale, dt, dt_u, heads=heads)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    n_kv = res["n_q"] + res["n_cache"]
+    flops = attention_flops(res["n_q"], n_kv, heads, wl.head_dim)
+    return flops, float(np.mean(times))
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        n = 1
+    try:
+        n = min(n, len(os.sched_getaffinity(0)))
+    except Exception:
+        pass
+    return int(n)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = args.config
+    wl, lat, qkv = make_workload(cfg, 0)
+    heads = wl.heads
+    steps = 3 if args.steps is None else max(1, min(args.steps, 20))
+    warmup = 1 if args.warmup is None else max(0, min(args.warmup, 3))
+    flops, sec = time_oracle(wl, lat, qkv, heads, steps, warmup)
+    val = flops / sec / 1e12
+    cores = host_threads()
+    sample = (f"whole step on config {cfg} ({wl.name}) with the attention restricted to {heads} of "
+              f"{wl.heads} heads; all other stages at full size")
+    line = dict(metric=METRIC, value=val, unit=UNIT, impl="reference", n_gpus=args.gpus, steps=steps,
+                warmup=warmup, ms_per_step=sec * 1e3, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=f"config {cfg}: {wl.name}", sample=sample),
+                cpu_baseline=dict(value=val, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=val, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2510_25590_b200 import binding, build as _build, synth
+    from paper_2510_25590_b200.step import RegionStep, StepShapes, plan_capacity
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    binding.load()
+
+    steps = 1000 if args.steps is None else args.steps
+    warmup = 10 if args.warmup is None else max(3, args.warmup)
+    cfg = args.config
+    # weak scaling: every rank owns its own request(s) (a different seed stream), no exchange
+    wl, lat, qkv = make_workload(cfg, shard_requests(world, world, rank)[0])
+    bf = torch.bfloat16
+
+    def dev(a):
+        bits = synth.f32_to_bf16_bits(a).reshape(a.shape)
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(bf)
+
+    def pinned(a):
+        bits = synth.f32_to_bf16_bits(a).reshape(a.shape)
+        return torch.from_numpy(bits.view(np.int16)).view(bf).pin_memory()
+
+    host = {k: pinned(v) for k, v in (("x_t", lat["x_t"]), ("v", lat["v"]), ("ref", lat["ref"]),
+                                      ("q", qkv["q"]), ("k", qkv["k"]), ("vv", qkv["v"]))}
+    d = {k: v.cuda() for k, v in host.items()}
+    t, scale, dt, dt_u = lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0
+    metric = binding.METRIC_COSINE if wl.metric == "cosine" else binding.METRIC_L2
+    cap = plan_capacity(d["x_t"], d["v"], d["ref"], t, metric, wl.threshold)
+    shp = StepShapes(wl.batch, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads, wl.head_dim, cap,
+                     metric, wl.threshold)
+    step = RegionStep(shp)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
+
+    def one():
+        step.run(d["x_t"], d["v"], d["ref"], d["q"], d["k"], d["vv"], t, scale, dt, dt_u)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    assert int(step.dev_status[0]) == 0, binding.status_string(int(step.dev_status[0]))
+    n_q = step.n_q.cpu().numpy()
+    n_kv = n_q + step.n_cache.cpu().numpy()
+    flops = attention_flops(n_q, n_kv, wl.heads, wl.head_dim)
+
+    # ---- timed region: K steps, L2 flushed before each, per-step and per-attention events ----
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    aev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    sampler = ClockSampler(local)
+    launches0 = step.launches
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    wall0 = time.perf_counter()
+    for i in range(steps):
+        flush.zero_()
+        step.attention_events = aev[i]
+        ev[i][0].record()
+        one()
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop()
+    step.attention_events = None
+    launches = step.launches - launches0
+    step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    attn_ms = np.array([a.elapsed_time(b) for a, b in aev])
+    total_ms = float(step_ms.sum())
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / steps
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: pinned host inputs -> device, the step, result -> host, every step ----
+    e2e_steps = max(3, min(steps, 50))
+    out_host = torch.empty_like(step.x_out, device="cpu").pin_memory()
+    o_host = torch.empty_like(step.o_e, device="cpu").pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = out_host.numel() * 2 + o_host.numel() * 2
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def one_e2e():
+        for k in host:
+            d[k].copy_(host[k], non_blocking=True)
+        one()
+        out_host.copy_(step.x_out, non_blocking=True)
+        o_host.copy_(step.o_e, non_blocking=True)
+
+    for _ in range(2):
+        one_e2e()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        one_e2e()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        tt = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_val = world * flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    attn_us = float(np.mean(attn_ms) * 1e3)
+    achieved = flops / (attn_us * 1e-6) / 1e12
+    roofline = dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                    frac=achieved / peaks["bf16_tflops"], traffic=recorded_traffic(),
+                    kernel="region_attention_tc_kernel<128>", us_per_launch=attn_us,
+                    peak_source=f"bf16_tflops (burst) of {peaks['source']}",
+                    frac_of_nominal_2250=achieved / NOMINAL_BF16_TFLOPS)
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        heads = wl.heads
+        fl, sec = time_oracle(wl, lat, qkv, heads, 2, 1)
+        cpu_baseline = dict(value=fl / sec / 1e12, unit=UNIT, cores=host_threads(), kind="oracle",
+                            sample=f"whole step on config {cfg} with the attention restricted to {heads} of "
+                                   f"{wl.heads} heads ({sec:.2f} s per step); other stages at full size")
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps, warmup=warmup,
+                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16", data="synthetic",
+                config=dict(workload=f"config {cfg}: {wl.name}", batch=wl.batch, image_tokens=wl.n_img,
+                            reference_tokens=wl.n_ref, text_tokens=wl.n_text, heads=wl.heads,
+                            head_dim=wl.head_dim, n_q=int(n_q[0]), n_kv=int(n_kv[0]),
+                            cache_policy="L2 flushed (256 MiB memset) before every timed step",
+                            parallelism=f"replicas x{world} (independent requests, no collective)"),
+                clocks=clocks,
+                e2e=dict(value=e2e_val, unit=UNIT, h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=int(d2h),
+                         steps=e2e_steps, ms_per_step=e2e_ms / e2e_steps),
+                gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu_baseline,
+                step_us=dict(mean=float(step_ms.mean() * 1e3), min=float(step_ms.min() * 1e3),
+                             median=float(np.median(step_ms) * 1e3)),
+                attention_us=dict(mean=attn_us, min=float(attn_ms.min() * 1e3)),
+                wall_s_timed_region=wall)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 5])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

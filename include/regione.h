@@ -1,0 +1,227 @@
+/*
+ * regione.h -- C ABI of libregione.so: the region-aware denoising step of a
+ * flow-matching DiT image editor (RegionE, arXiv 2510.25590), as hand-written
+ * CUDA kernels for sm_100a (NVIDIA B200).
+ *
+ * Conventions
+ * -----------
+ *  - Every function returns a regione_status.  Argument validation is done
+ *    synchronously on the host; the work itself is enqueued on `stream`
+ *    (a cudaStream_t passed as void*, NULL = default stream) and is
+ *    asynchronous.  Nothing synchronises the device.
+ *  - "dev" pointers are device memory owned by the caller; "host" values are
+ *    plain scalars.  Unless a function says otherwise the library allocates
+ *    nothing and keeps no state between calls.
+ *  - bf16 tensors are passed as regione_bf16* (raw bfloat16 bit patterns),
+ *    row-major with the last index contiguous.  All bf16 tensors must be
+ *    16-byte aligned.  Arithmetic is fp32; results are rounded to bf16 with
+ *    round-to-nearest-even.
+ *  - Per-request counts (n_edit, n_q, ...) live in device memory as int32 so
+ *    that no host round trip is needed between the partition and the calls
+ *    that consume its output; capacities (*_cap) are host ints.
+ *  - `dev_status` (nullable, device int32, caller zeroes it) receives
+ *    REGIONE_DEV_BOUNDS or REGIONE_DEV_TIMEOUT if a kernel meets an index or
+ *    count outside its capacity or a bounded wait runs out.  Kernels never
+ *    trap: the offending access is skipped and the kernel ends normally.
+ *  - B is the number of independent edit requests in the batch; they share
+ *    the sampler schedule (t, dt, scale are scalars).
+ *  - There is no CPU fallback: without a CUDA device every compute entry point
+ *    returns REGIONE_CUDA_ERROR.
+ */
+#ifndef REGIONE_H_
+#define REGIONE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t regione_bf16;
+
+typedef enum {
+    REGIONE_OK = 0,
+    REGIONE_INVALID_ARG = 1,        /* null pointer, negative size, misaligned pointer */
+    REGIONE_UNSUPPORTED = 2,        /* shape outside what the kernels implement */
+    REGIONE_CUDA_ERROR = 3,         /* a CUDA runtime/driver call failed (launch, tensor map) */
+    REGIONE_WORKSPACE_TOO_SMALL = 4
+} regione_status;
+
+enum { REGIONE_DEV_OK = 0, REGIONE_DEV_TIMEOUT = 5, REGIONE_DEV_BOUNDS = 6 };
+
+enum { REGIONE_METRIC_COSINE = 0, REGIONE_METRIC_L2 = 1 };
+
+/* membership of the joint sequence rows in one region-attention call */
+enum { REGIONE_ROWS_EDITED_QUERIES = 0, REGIONE_ROWS_PAPER = 1 };
+
+/* Library version (major*10000 + minor*100 + patch) and status names. */
+int regione_version(void);
+const char* regione_status_string(int status);
+
+/*
+ * Adaptive Region Partition (Sec. 4, "Adaptive Region Partition"; Algorithm 1,
+ * the two lines computing X_hat_0 and E_index/U_index), without the
+ * morphological clean-up.
+ *
+ * For every request b and token n:
+ *     x0_hat[c] = x_t[b,n,c] - t * v[b,n,c]                (one-step estimate, t_f = 0)
+ *     s = cos(x0_hat, ref[b,n,:])      (metric COSINE;  edited iff s <= threshold)
+ *     s = || x0_hat - ref[b,n,:] ||_2  (metric L2;      edited iff s >  threshold)
+ * and then, per request, the ascending index lists:
+ *     edit_idx[b, 0..n_edit[b])      token ids with mask = 1
+ *     keep_idx[b, 0..N-n_edit[b])    token ids with mask = 0
+ *     slot[b,n] = position of n in edit_idx, or -1
+ * A zero cosine denominator is clamped at 1e-12.
+ *
+ * x_t, v, ref : dev bf16 [B, N, C], C a multiple of 8 and <= 4096
+ * mask        : dev u8    [B, N]   (1 = edited)
+ * edit_idx, keep_idx, slot : dev int32 [B, N]; entries of edit_idx / keep_idx past
+ *               the live prefix are left untouched
+ * n_edit      : dev int32 [B]
+ * score       : dev f32   [B, N], nullable; receives s
+ * Limits: 1 <= N <= 2^21 per request, B <= 65535.
+ */
+int regione_partition(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
+                      int B, int N, int C, float t, int metric, float threshold,
+                      uint8_t* mask, int32_t* edit_idx, int32_t* keep_idx, int32_t* slot,
+                      int32_t* n_edit, float* score, int32_t* dev_status, void* stream);
+
+/*
+ * Morphological opening then closing of the edited mask on the rows x cols token
+ * grid (Sec. 4, "Adaptive Region Partition": "morphological opening and closing
+ * operations"; Algorithm 1 calls it Erosion_&_Dilate), followed by the same
+ * compaction as regione_partition.  Structuring element 3x3; neighbours outside
+ * the grid are ignored.  mask_in [B, rows*cols] -> mask_out and the index lists.
+ * mask_in and mask_out may not alias.  rows*cols <= 16384.
+ */
+int regione_mask_open_close(const uint8_t* mask_in, int B, int rows, int cols,
+                            uint8_t* mask_out, int32_t* edit_idx, int32_t* keep_idx,
+                            int32_t* slot, int32_t* n_edit, int32_t* dev_status, void* stream);
+
+/*
+ * Joint-sequence row lists for one region-attention layer, composed on the
+ * device from the partition's output (Sec. 4, "Region-Aware Generation": which
+ * tokens are recomputed and which come from the cache).  The joint sequence is
+ * [text (n_text) | image (N) | reference (n_ref)].
+ *   REGIONE_ROWS_EDITED_QUERIES: query_rows = n_text + edit_idx;
+ *        cache_rows = text, n_text + keep_idx, reference   (ascending)
+ *   REGIONE_ROWS_PAPER: query_rows = text, n_text + edit_idx;
+ *        cache_rows = n_text + keep_idx, reference
+ * query_rows : dev int32 [B, q_cap],  n_query dev int32 [B]
+ * cache_rows : dev int32 [B, c_cap],  n_cache dev int32 [B]
+ * Counts beyond a capacity are clamped and REGIONE_DEV_BOUNDS is recorded.
+ */
+int regione_region_rows(const int32_t* edit_idx, const int32_t* keep_idx, const int32_t* n_edit,
+                        int B, int N, int n_text, int n_ref, int membership,
+                        int32_t* query_rows, int32_t* n_query, int q_cap,
+                        int32_t* cache_rows, int32_t* n_cache, int c_cap,
+                        int32_t* dev_status, void* stream);
+
+/*
+ * Token gather (Algorithm 1: X^E = X[E_index], X^U = X[U_index]):
+ *     dst[b, j, :] = src[b, idx[b, j], :]     for j < min(n[b], dst_rows_cap)
+ * Rows are opaque byte strings of row_bytes (a multiple of 16) bytes.
+ * src [B, src_rows, row_bytes], idx dev int32 [B, idx_stride], n dev int32 [B],
+ * dst [B, dst_rows_cap, row_bytes].  Rows of dst past n[b] are left untouched.
+ * An index outside [0, src_rows) is skipped and REGIONE_DEV_BOUNDS recorded.
+ */
+int regione_gather(const void* src, const int32_t* idx, const int32_t* n, int B,
+                   int64_t src_rows, int64_t idx_stride, int64_t dst_rows_cap, int64_t row_bytes,
+                   void* dst, int32_t* dev_status, void* stream);
+
+/*
+ * Token scatter, the inverse placement (Sec. 4: results are "re-gathered according
+ * to their spatial positions"; Algorithm 1, the gather(...) line):
+ *     dst[b, idx[b, j], :] = src[b, j, :]     for j < min(n[b], src_rows_cap)
+ * Other rows of dst are left untouched.  idx must not repeat a row.
+ */
+int regione_scatter(const void* src, const int32_t* idx, const int32_t* n, int B,
+                    int64_t src_rows_cap, int64_t idx_stride, int64_t dst_rows, int64_t row_bytes,
+                    void* dst, int32_t* dev_status, void* stream);
+
+/*
+ * Region-Instruction KV cache store (Sec. 4, "Stabilization Stage": the Key and
+ * Value of each attention layer are saved at the last full step; refreshed at
+ * forced steps).  Compacts the retained rows of one layer's full K and V:
+ *     k_cache[b, j, :, :] = k_full[b, keep_rows[b, j], :, :]   (same for V),  j < n_keep[b]
+ * k_full, v_full [B, N_full, H, D] bf16; keep_rows dev int32 [B, Nc_cap];
+ * k_cache, v_cache [B, Nc_cap, H, D].  H*D must be a multiple of 8.
+ */
+int regione_rikv_store(const regione_bf16* k_full, const regione_bf16* v_full,
+                       const int32_t* keep_rows, const int32_t* n_keep,
+                       int B, int N_full, int Nc_cap, int H, int D,
+                       regione_bf16* k_cache, regione_bf16* v_cache,
+                       int32_t* dev_status, void* stream);
+
+/*
+ * Region attention with the Region-Instruction KV cache (Sec. 4, "Region-Aware
+ * Generation", the attention equation):
+ *     out[b,i,h,:] = sum_j softmax_j( scale * q[b,i,h,:] . k_j ) * v_j
+ * with j running over the fresh rows 0..n_fresh[b) of (k_fresh, v_fresh) and the
+ * cached rows 0..n_cache[b) of (k_cache, v_cache); the concatenation is never
+ * materialised.  No mask, no positional encoding (the cache holds K as it
+ * entered the softmax at the storing step).
+ *
+ * q, out          : dev bf16 [B, Nq_cap, H, D];  rows i >= n_q[b] are not written
+ * k_fresh, v_fresh: dev bf16 [B, Nf_cap, H, D]
+ * k_cache, v_cache: dev bf16 [B, Nc_cap, H, D]   (may be NULL when Nc_cap == 0)
+ * n_q, n_fresh, n_cache : dev int32 [B]; values above the capacity are clamped and
+ *                   REGIONE_DEV_BOUNDS recorded
+ * softmax_scale   : <= 0 selects 1/sqrt(D)
+ * workspace       : dev, 256-byte aligned, at least
+ *                   regione_region_attention_workspace(...) bytes (may be 0 -> NULL ok)
+ * D must be 64 or 128.  bf16 inputs, fp32 accumulation, probabilities rounded
+ * to bf16 before the second product.  With no key at all a row is zero.
+ */
+size_t regione_region_attention_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D);
+int regione_region_attention(const regione_bf16* q,
+                             const regione_bf16* k_fresh, const regione_bf16* v_fresh,
+                             const regione_bf16* k_cache, const regione_bf16* v_cache,
+                             const int32_t* n_q, const int32_t* n_fresh, const int32_t* n_cache,
+                             int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D,
+                             float softmax_scale, regione_bf16* out,
+                             void* workspace, size_t workspace_bytes,
+                             int32_t* dev_status, void* stream);
+
+/*
+ * One step of the AVDCache criterion (Sec. 4, "Adaptive Velocity Decay Cache",
+ * the decay-factor and criterion equations).  Pure host arithmetic:
+ *     p = *running_product * (1 - dt) * gamma
+ *     if 1 - p > delta : *reuse = 0, *running_product = 1     (recompute, refresh the cache)
+ *     else             : *reuse = 1, *running_product = p     (use cached velocity * p)
+ */
+int regione_avd_step(double* running_product, double dt, double gamma, double delta, int* reuse);
+
+/*
+ * Decayed cached velocity and Euler update of the edited tokens (Sec. 4, the
+ * case equation of the AVDCache; Sec. 3, the Euler sampler equation):
+ *     v_use = scale * v_in[b,j,:]
+ *     x_e[b,j,:] <- x_e[b,j,:] - dt * v_use                for j < n_edit[b]
+ *     v_cache_out[b,j,:] <- v_in[b,j,:]   (if v_cache_out != NULL: a recomputed step
+ *                                          refreshes the velocity cache)
+ * scale is the accumulated decay product on a reused step and 1 on a recomputed one.
+ * v_in, x_e, v_cache_out : dev bf16 [B, Ne_cap, C], C a multiple of 8.
+ */
+int regione_velocity_decay(const regione_bf16* v_in, float scale, float dt, regione_bf16* x_e,
+                           regione_bf16* v_cache_out, const int32_t* n_edit,
+                           int B, int Ne_cap, int C, int32_t* dev_status, void* stream);
+
+/*
+ * Merge of the two regions at the end of a run of region steps (Sec. 4, one-step
+ * estimation equation applied to the unedited tokens; Algorithm 1, the one-step
+ * line before the inner loop and the gather line after it):
+ *     x_out[b,n,:] = slot[b,n] >= 0 ? x_e[b, slot[b,n], :]
+ *                                   : x_full[b,n,:] - dt_unedited * v_last_full[b,n,:]
+ * x_full, v_last_full, x_out : dev bf16 [B, N, C]; x_e [B, Ne_cap, C]; slot dev int32 [B, N].
+ * x_out may alias x_full.  A slot >= Ne_cap is skipped and REGIONE_DEV_BOUNDS recorded.
+ */
+int regione_merge(const regione_bf16* x_full, const regione_bf16* v_last_full,
+                  const regione_bf16* x_e, const int32_t* slot, float dt_unedited,
+                  int B, int N, int Ne_cap, int C, regione_bf16* x_out,
+                  int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REGIONE_H_ */

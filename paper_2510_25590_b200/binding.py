@@ -1,0 +1,228 @@
+"""ctypes binding over the C ABI of ``libregione.so`` (see ``include/regione.h``).
+
+Argument marshalling only: every function takes torch CUDA tensors (used purely
+as device buffers), checks dtype / contiguity, and forwards raw pointers and
+sizes to the entry point of the same name.  There is no fallback of any kind:
+if the shared library is missing or a call fails, a ``RegionEError`` is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, c_char_p, c_double, c_float, c_int, c_int64, c_size_t, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libregione.so")
+
+OK, INVALID_ARG, UNSUPPORTED, CUDA_ERROR, WORKSPACE_TOO_SMALL = 0, 1, 2, 3, 4
+DEV_OK, DEV_TIMEOUT, DEV_BOUNDS = 0, 5, 6
+METRIC_COSINE, METRIC_L2 = 0, 1
+ROWS_EDITED_QUERIES, ROWS_PAPER = 0, 1
+
+# every symbol include/regione.h declares: name -> (restype, argtypes)
+_P = c_void_p
+SIGNATURES = {
+    "regione_version": (c_int, []),
+    "regione_status_string": (c_char_p, [c_int]),
+    "regione_partition": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_float, c_int, c_float,
+                                  _P, _P, _P, _P, _P, _P, _P, _P]),
+    "regione_mask_open_close": (c_int, [_P, c_int, c_int, c_int, _P, _P, _P, _P, _P, _P, _P]),
+    "regione_region_rows": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_int, c_int,
+                                    _P, _P, c_int, _P, _P, c_int, _P, _P]),
+    "regione_gather": (c_int, [_P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int64, _P, _P, _P]),
+    "regione_scatter": (c_int, [_P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int64, _P, _P, _P]),
+    "regione_rikv_store": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
+    "regione_region_attention_workspace": (c_size_t, [c_int] * 6),
+    "regione_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, c_size_t, _P, _P]),
+    "regione_avd_step": (c_int, [POINTER(c_double), c_double, c_double, c_double, POINTER(c_int)]),
+    "regione_velocity_decay": (c_int, [_P, c_float, c_float, _P, _P, _P, c_int, c_int, c_int, _P, _P]),
+    "regione_merge": (c_int, [_P, _P, _P, _P, c_float, c_int, c_int, c_int, c_int, _P, _P, _P]),
+}
+
+
+class RegionEError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load(path: str | None = None) -> ctypes.CDLL:
+    """Loads libregione.so (once) and declares every entry point.  Raises if it is missing."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise RegionEError(
+            f"{p} not found: build it with `python -m paper_2510_25590_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(p)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load().regione_status_string(int(code)).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != OK:
+        raise RegionEError(f"{what} failed: {status_string(code)} ({code})")
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _ptr(t, dtype=None, name="tensor"):
+    if t is None:
+        return None
+    torch = _torch()
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise RegionEError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise RegionEError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise RegionEError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    return c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    torch = _torch()
+    s = torch.cuda.current_stream() if stream is None else stream
+    return c_void_p(s.cuda_stream)
+
+
+def version() -> int:
+    return load().regione_version()
+
+
+def partition(x_t, v, ref, t, metric, threshold, mask, edit_idx, keep_idx, slot, n_edit,
+              score=None, dev_status=None, stream=None):
+    torch = _torch()
+    B, N, C = x_t.shape
+    bf = torch.bfloat16
+    _check(load().regione_partition(
+        _ptr(x_t, bf, "x_t"), _ptr(v, bf, "v"), _ptr(ref, bf, "ref"), B, N, C, float(t), int(metric),
+        float(threshold), _ptr(mask, torch.uint8, "mask"), _ptr(edit_idx, torch.int32, "edit_idx"),
+        _ptr(keep_idx, torch.int32, "keep_idx"), _ptr(slot, torch.int32, "slot"),
+        _ptr(n_edit, torch.int32, "n_edit"), _ptr(score, torch.float32, "score"),
+        _ptr(dev_status, torch.int32, "dev_status"), _stream(stream)), "regione_partition")
+
+
+def mask_open_close(mask_in, rows, cols, mask_out, edit_idx, keep_idx, slot, n_edit,
+                    dev_status=None, stream=None):
+    torch = _torch()
+    B = mask_in.shape[0]
+    _check(load().regione_mask_open_close(
+        _ptr(mask_in, torch.uint8, "mask_in"), B, int(rows), int(cols),
+        _ptr(mask_out, torch.uint8, "mask_out"), _ptr(edit_idx, torch.int32), _ptr(keep_idx, torch.int32),
+        _ptr(slot, torch.int32), _ptr(n_edit, torch.int32), _ptr(dev_status, torch.int32),
+        _stream(stream)), "regione_mask_open_close")
+
+
+def region_rows(edit_idx, keep_idx, n_edit, n_text, n_ref, membership, query_rows, n_query,
+                cache_rows, n_cache, dev_status=None, stream=None):
+    torch = _torch()
+    B, N = edit_idx.shape
+    i32 = torch.int32
+    _check(load().regione_region_rows(
+        _ptr(edit_idx, i32), _ptr(keep_idx, i32), _ptr(n_edit, i32), B, N, int(n_text), int(n_ref),
+        int(membership), _ptr(query_rows, i32), _ptr(n_query, i32), query_rows.shape[1],
+        _ptr(cache_rows, i32), _ptr(n_cache, i32), cache_rows.shape[1], _ptr(dev_status, i32),
+        _stream(stream)), "regione_region_rows")
+
+
+def _row_bytes(t):
+    rb = t.element_size()
+    for d in t.shape[2:]:
+        rb *= d
+    return rb
+
+
+def gather(src, idx, n, dst, dev_status=None, stream=None):
+    """dst[b, j] = src[b, idx[b, j]], j < n[b].  src [B, rows, ...], dst [B, cap, ...]."""
+    torch = _torch()
+    B = src.shape[0]
+    _check(load().regione_gather(
+        _ptr(src, None, "src"), _ptr(idx, torch.int32, "idx"), _ptr(n, torch.int32, "n"), B,
+        src.shape[1], idx.shape[1], dst.shape[1], _row_bytes(src), _ptr(dst, src.dtype, "dst"),
+        _ptr(dev_status, torch.int32), _stream(stream)), "regione_gather")
+
+
+def scatter(src, idx, n, dst, dev_status=None, stream=None):
+    """dst[b, idx[b, j]] = src[b, j], j < n[b].  src [B, cap, ...], dst [B, rows, ...]."""
+    torch = _torch()
+    B = src.shape[0]
+    _check(load().regione_scatter(
+        _ptr(src, None, "src"), _ptr(idx, torch.int32, "idx"), _ptr(n, torch.int32, "n"), B,
+        src.shape[1], idx.shape[1], dst.shape[1], _row_bytes(src), _ptr(dst, src.dtype, "dst"),
+        _ptr(dev_status, torch.int32), _stream(stream)), "regione_scatter")
+
+
+def rikv_store(k_full, v_full, keep_rows, n_keep, k_cache, v_cache, dev_status=None, stream=None):
+    torch = _torch()
+    bf = torch.bfloat16
+    B, n_full, H, D = k_full.shape
+    _check(load().regione_rikv_store(
+        _ptr(k_full, bf, "k_full"), _ptr(v_full, bf, "v_full"), _ptr(keep_rows, torch.int32),
+        _ptr(n_keep, torch.int32), B, n_full, k_cache.shape[1], H, D, _ptr(k_cache, bf, "k_cache"),
+        _ptr(v_cache, bf, "v_cache"), _ptr(dev_status, torch.int32), _stream(stream)),
+        "regione_rikv_store")
+
+
+def region_attention_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D) -> int:
+    return int(load().regione_region_attention_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D))
+
+
+def region_attention(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, out,
+                     softmax_scale=0.0, workspace=None, dev_status=None, stream=None):
+    torch = _torch()
+    bf = torch.bfloat16
+    B, Nq_cap, H, D = q.shape
+    Nf_cap = 0 if k_fresh is None else k_fresh.shape[1]
+    Nc_cap = 0 if k_cache is None else k_cache.shape[1]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    i32 = torch.int32
+    _check(load().regione_region_attention(
+        _ptr(q, bf, "q"), _ptr(k_fresh, bf, "k_fresh"), _ptr(v_fresh, bf, "v_fresh"),
+        _ptr(k_cache, bf, "k_cache"), _ptr(v_cache, bf, "v_cache"), _ptr(n_q, i32), _ptr(n_fresh, i32),
+        _ptr(n_cache, i32), B, Nq_cap, Nf_cap, Nc_cap, H, D, float(softmax_scale), _ptr(out, bf, "out"),
+        _ptr(workspace, None, "workspace"), ws_bytes, _ptr(dev_status, i32), _stream(stream)),
+        "regione_region_attention")
+
+
+def avd_step(running_product: float, dt: float, gamma: float, delta: float):
+    """Returns (new_running_product, reuse)."""
+    p = c_double(running_product)
+    r = c_int(0)
+    _check(load().regione_avd_step(ctypes.byref(p), dt, gamma, delta, ctypes.byref(r)),
+           "regione_avd_step")
+    return p.value, bool(r.value)
+
+
+def velocity_decay(v_in, scale, dt, x_e, n_edit, v_cache_out=None, dev_status=None, stream=None):
+    torch = _torch()
+    bf = torch.bfloat16
+    B, Ne_cap, C = x_e.shape
+    _check(load().regione_velocity_decay(
+        _ptr(v_in, bf, "v_in"), float(scale), float(dt), _ptr(x_e, bf, "x_e"),
+        _ptr(v_cache_out, bf, "v_cache_out"), _ptr(n_edit, torch.int32), B, Ne_cap, C,
+        _ptr(dev_status, torch.int32), _stream(stream)), "regione_velocity_decay")
+
+
+def merge(x_full, v_last_full, x_e, slot, dt_unedited, x_out, dev_status=None, stream=None):
+    torch = _torch()
+    bf = torch.bfloat16
+    B, N, C = x_full.shape
+    _check(load().regione_merge(
+        _ptr(x_full, bf, "x_full"), _ptr(v_last_full, bf, "v_last_full"), _ptr(x_e, bf, "x_e"),
+        _ptr(slot, torch.int32), float(dt_unedited), B, N, 0 if x_e is None else x_e.shape[1], C,
+        _ptr(x_out, bf, "x_out"), _ptr(dev_status, torch.int32), _stream(stream)), "regione_merge")

@@ -1,0 +1,94 @@
+// Host-only entry points of libregione: version, status names, the AVDCache
+// criterion (a scalar recurrence evaluated on the host), and the dispatcher of
+// the region attention.
+#include <cstdlib>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace regione {
+int launch_region_attention_simt(const uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*,
+                                 const uint16_t*, const int32_t*, const int32_t*, const int32_t*,
+                                 int, int, int, int, int, int, float, uint16_t*, int32_t*,
+                                 cudaStream_t);
+size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D);
+int launch_region_attention_tc(const uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*,
+                               const uint16_t*, const int32_t*, const int32_t*, const int32_t*, int,
+                               int, int, int, int, int, float, uint16_t*, void*, size_t, int32_t*,
+                               cudaStream_t);
+}  // namespace regione
+
+using namespace regione;
+
+extern "C" int regione_version(void) { return 100; }
+
+extern "C" const char* regione_status_string(int status) {
+    switch (status) {
+        case REGIONE_OK: return "REGIONE_OK";
+        case REGIONE_INVALID_ARG: return "REGIONE_INVALID_ARG";
+        case REGIONE_UNSUPPORTED: return "REGIONE_UNSUPPORTED";
+        case REGIONE_CUDA_ERROR: return "REGIONE_CUDA_ERROR";
+        case REGIONE_WORKSPACE_TOO_SMALL: return "REGIONE_WORKSPACE_TOO_SMALL";
+        case REGIONE_DEV_TIMEOUT: return "REGIONE_DEV_TIMEOUT";
+        case REGIONE_DEV_BOUNDS: return "REGIONE_DEV_BOUNDS";
+        default: return "REGIONE_UNKNOWN";
+    }
+}
+
+extern "C" int regione_avd_step(double* running_product, double dt, double gamma, double delta,
+                                int* reuse) {
+    if (!running_product || !reuse) return REGIONE_INVALID_ARG;
+    const double p = *running_product * (1.0 - dt) * gamma;
+    if (1.0 - p > delta) {
+        *reuse = 0;
+        *running_product = 1.0;
+    } else {
+        *reuse = 1;
+        *running_product = p;
+    }
+    return REGIONE_OK;
+}
+
+static bool use_simt() {
+    const char* e = std::getenv("REGIONE_ATTENTION_IMPL");
+    return e != nullptr && std::strcmp(e, "simt") == 0;
+}
+
+extern "C" size_t regione_region_attention_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap,
+                                                     int H, int D) {
+    if (B <= 0 || Nq_cap <= 0 || H <= 0 || (D != 64 && D != 128)) return 0;
+    return region_attention_tc_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D);
+}
+
+extern "C" int regione_region_attention(const regione_bf16* q, const regione_bf16* k_fresh,
+                                        const regione_bf16* v_fresh, const regione_bf16* k_cache,
+                                        const regione_bf16* v_cache, const int32_t* n_q,
+                                        const int32_t* n_fresh, const int32_t* n_cache, int B,
+                                        int Nq_cap, int Nf_cap, int Nc_cap, int H, int D,
+                                        float softmax_scale, regione_bf16* out, void* workspace,
+                                        size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    if (!q || !out || !n_q || !n_fresh || !n_cache) return REGIONE_INVALID_ARG;
+    if (B < 0 || Nq_cap < 0 || Nf_cap < 0 || Nc_cap < 0 || H < 1) return REGIONE_INVALID_ARG;
+    if (Nf_cap > 0 && (!k_fresh || !v_fresh)) return REGIONE_INVALID_ARG;
+    if (Nc_cap > 0 && (!k_cache || !v_cache)) return REGIONE_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_fresh) || !aligned16(v_fresh) ||
+        !aligned16(k_cache) || !aligned16(v_cache))
+        return REGIONE_INVALID_ARG;
+    if (D != 64 && D != 128) return REGIONE_UNSUPPORTED;
+    if (B > 65535 || H > 65535) return REGIONE_UNSUPPORTED;
+    if (B == 0 || Nq_cap == 0) return REGIONE_OK;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (use_simt())
+        return launch_region_attention_simt(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh,
+                                            n_cache, B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out,
+                                            dev_status, st);
+    const size_t need = region_attention_tc_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D);
+    if (need > 0) {
+        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return REGIONE_INVALID_ARG;
+        if (workspace_bytes < need) return REGIONE_WORKSPACE_TOO_SMALL;
+    }
+    return launch_region_attention_tc(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
+                                      B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, workspace,
+                                      workspace_bytes, dev_status, st);
+}

@@ -1,0 +1,451 @@
+// Region attention with the Region-Instruction KV cache on the 5th-generation
+// tensor cores (Sec. 4 "Region-Aware Generation", the attention equation):
+// queries of the recomputed tokens against [fresh keys | cached keys] without
+// materialising the concatenation.
+//
+// One CTA = one (request, head, pair of 128-row query tiles).  Warp roles:
+//   warps 0-3  softmax / correction / epilogue of query tile 0 (thread = row)
+//   warps 4-7  the same for query tile 1
+//   warp  8    TMA producer: Q once, then K_j, V_j tiles through a ring of
+//              shared-memory stages; the cached segment and the fresh segment
+//              are two tensor maps walked one after the other
+//   warp  9    tcgen05.mma issuer and owner of the tensor-memory allocation
+// Tensor memory (512 columns): S0 | S1 | O0 | O1.  S_t = Q_t K_j^T (fp32) is
+// read back by the softmax warps, the probabilities are written over it as
+// bf16 (P aliases S) and feed O_t += P_t V_j straight from tensor memory.
+// Online softmax in the exp2 domain; O is rescaled in tensor memory only when
+// a row maximum grows.  Rows past a segment's live count are masked in the
+// softmax and their V rows zeroed in shared memory, so garbage (even NaN)
+// behind the live prefix cannot leak.
+//
+// Every wait is bounded: if a barrier does not complete within ~2 s the CTA
+// records REGIONE_DEV_TIMEOUT, all roles leave their loops, tensor memory is
+// released and the kernel ends normally.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace regione {
+
+constexpr int kAttnThreads = 320;
+constexpr int kBM = 128;                 // query rows per tile
+constexpr int kBN = 128;                 // key rows per tile
+constexpr int kHalfBytes = 128 * 64 * 2; // one 128-row x 64-column bf16 box (128-byte rows)
+constexpr long long kTimeoutCycles = 4000000000LL;
+
+template <int D>
+struct AttnCfg {
+    static constexpr int kHalves = D / 64;
+    static constexpr int kTileBytes = kHalves * kHalfBytes;
+    static constexpr int kStages = (D == 128) ? 4 : 6;
+    static constexpr int kSmemTiles = (2 + kStages) * kTileBytes;
+    static constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 256 /*control*/;
+};
+
+struct AttnCtrl {
+    uint64_t q_full;
+    uint64_t kv_full[6];
+    uint64_t kv_empty[6];
+    uint64_t s_full[2];
+    uint64_t p_full[2];
+    uint64_t o_done[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct AttnParams {
+    const int32_t* n_q;
+    const int32_t* n_fresh;
+    const int32_t* n_cache;
+    int Nq_cap, Nf_cap, Nc_cap, H;
+    float scale_log2e;
+    uint16_t* out;
+    int32_t* dev_status;
+};
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                         int32_t* dev_status) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kTimeoutCycles) {
+            *abort_flag = 1;
+            record_status(dev_status, REGIONE_DEV_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
+                           const __grid_constant__ CUtensorMap tm_kf,
+                           const __grid_constant__ CUtensorMap tm_vf,
+                           const __grid_constant__ CUtensorMap tm_kc,
+                           const __grid_constant__ CUtensorMap tm_vc, const AttnParams p) {
+    using Cfg = AttnCfg<D>;
+    constexpr int kStages = Cfg::kStages;
+    constexpr int kTileBytes = Cfg::kTileBytes;
+
+    const int b = blockIdx.z, h = blockIdx.y;
+    const int q0 = blockIdx.x * (2 * kBM);
+    int nq = p.n_q[b], nf = p.n_fresh[b], nc = p.n_cache[b];
+    if (nq < 0 || nq > p.Nq_cap || nf < 0 || nf > p.Nf_cap || nc < 0 || nc > p.Nc_cap) {
+        if (threadIdx.x == 0) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+        nq = max(0, min(nq, p.Nq_cap));
+        nf = max(0, min(nf, p.Nf_cap));
+        nc = max(0, min(nc, p.Nc_cap));
+    }
+    if (q0 >= nq) return;                               // uniform for the CTA
+    const int ntq = (nq - q0 > kBM) ? 2 : 1;            // live query tiles of this CTA
+    const int nt_c = (nc + kBN - 1) / kBN;
+    const int nt_f = (nf + kBN - 1) / kBN;
+    const int n_tiles = nt_c + nt_f;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
+    const uint32_t sQ = smem_base;                      // 2 query tiles
+    const uint32_t sKV = smem_base + 2 * kTileBytes;    // ring of K/V stages
+    AttnCtrl* ctrl = reinterpret_cast<AttnCtrl*>(smem_gen + Cfg::kSmemTiles);
+    volatile int* abort_flag = &ctrl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_addr(&ctrl->q_full), 1);
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_full[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_empty[s]), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t]), kBM);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->o_done[t]), 1);
+        }
+        ctrl->abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    if (warp == 9) {
+        ptx::tmem_alloc(ptx::smem_addr(&ctrl->tmem_base), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = ctrl->tmem_base;
+
+    // tile j -> (segment, first row, live rows)
+    auto tile_seg = [&](int j, bool& cached, int& row0, int& valid) {
+        cached = j < nt_c;
+        const int jj = cached ? j : j - nt_c;
+        row0 = jj * kBN;
+        valid = min(kBN, (cached ? nc : nf) - row0);
+    };
+
+    if (warp == 8) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            ptx::prefetch_tensormap(&tm_q);
+            ptx::prefetch_tensormap(nt_c ? &tm_kc : &tm_kf);
+            ptx::prefetch_tensormap(nt_c ? &tm_vc : &tm_vf);
+            const uint32_t qbar = ptx::smem_addr(&ctrl->q_full);
+            ptx::mbar_arrive_expect_tx(qbar, ntq * kTileBytes);
+            for (int t = 0; t < ntq; ++t)
+                for (int hf = 0; hf < Cfg::kHalves; ++hf)
+                    ptx::tma_load_4d(sQ + t * kTileBytes + hf * kHalfBytes, &tm_q, qbar, hf * 64, h,
+                                     q0 + t * kBM, b);
+            bool ok = true;
+            for (int i = 0; i < 2 * n_tiles && ok; ++i) {
+                const int j = i >> 1, is_v = i & 1;
+                const int stage = i % kStages, use = i / kStages;
+                if (use > 0)
+                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_empty[stage]), (use - 1) & 1, abort_flag,
+                                  p.dev_status);
+                if (!ok) break;
+                bool cached; int row0, valid;
+                tile_seg(j, cached, row0, valid);
+                const CUtensorMap* map = cached ? (is_v ? &tm_vc : &tm_kc) : (is_v ? &tm_vf : &tm_kf);
+                const uint32_t bar = ptx::smem_addr(&ctrl->kv_full[stage]);
+                ptx::mbar_arrive_expect_tx(bar, kTileBytes);
+                for (int hf = 0; hf < Cfg::kHalves; ++hf)
+                    ptx::tma_load_4d(sKV + stage * kTileBytes + hf * kHalfBytes, map, bar, hf * 64, h,
+                                     row0, b);
+            }
+        }
+    } else if (warp == 9) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
+            constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
+            // S_t = Q_t K^T : both operands K-major, 128-byte swizzle, 8-row groups 1024 B apart.
+            auto issue_s = [&](int t, int stage) {
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                    const uint64_t da = ptx::smem_desc_sw128(sQ + t * kTileBytes + off, 16, 1024);
+                    const uint64_t db = ptx::smem_desc_sw128(sKV + stage * kTileBytes + off, 16, 1024);
+                    ptx::mma_ss(tmem + t * kBN, da, db, idesc_s, kk > 0);
+                }
+            };
+            // O_t (+)= P_t V : A from tensor memory (bf16 pairs, 8 columns per 16 keys), B = V
+            // MN-major: 64-column boxes 16 KB apart (LBO), 8-key groups 1024 B apart (SBO).
+            auto issue_pv = [&](int t, int stage, bool accumulate) {
+#pragma unroll
+                for (int kk = 0; kk < kBN / 16; ++kk) {
+                    const uint64_t db =
+                        ptx::smem_desc_sw128(sKV + stage * kTileBytes + kk * 2048, kHalfBytes, 1024);
+                    ptx::mma_ts(tmem + 256 + t * D, tmem + t * kBN + kk * 8, db, idesc_pv,
+                                (accumulate || kk > 0) ? 1u : 0u);
+                }
+            };
+            bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
+            if (ok && n_tiles > 0) {
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[0]), 0, abort_flag, p.dev_status);
+                if (ok) {
+                    ptx::tc_fence_after_sync();
+                    for (int t = 0; t < ntq; ++t) {
+                        issue_s(t, 0);
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
+                    }
+                    ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[0]));
+                }
+            }
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int iv = 2 * j + 1, ik = 2 * j + 2;
+                const int sv = iv % kStages, sk = ik % kStages;
+                const bool more = (j + 1 < n_tiles);
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                              p.dev_status);
+                for (int t = 0; t < ntq && ok; ++t) {
+                    ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t]), j & 1, abort_flag, p.dev_status);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    issue_pv(t, sv, j > 0);
+                    ptx::mma_commit(ptx::smem_addr(&ctrl->o_done[t]));
+                    if (t == ntq - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sv]));
+                    if (more) {
+                        if (t == 0)
+                            ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / kStages) & 1,
+                                          abort_flag, p.dev_status);
+                        if (!ok) break;
+                        issue_s(t, sk);
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
+                        if (t == ntq - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk]));
+                    }
+                }
+            }
+        }
+    } else if (warp < 4 * ntq) {
+        // ================= softmax / correction / epilogue =================
+        const int t = warp >> 2;
+        const int row = ((warp & 3) << 5) + lane;                  // row of the query tile
+        const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
+        const uint32_t tS = tmem + lane_sel + t * kBN;
+        const uint32_t tO = tmem + lane_sel + 256 + t * D;
+        const float c = p.scale_log2e;
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        uint32_t r[32];
+        for (int j = 0; j < n_tiles; ++j) {
+            ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            bool cached; int row0, valid;
+            tile_seg(j, cached, row0, valid);
+            // pass 1: row maximum over the live columns
+            float mx = -INFINITY;
+#pragma unroll
+            for (int ch = 0; ch < kBN / 32; ++ch) {
+                ptx::tmem_ld32(tS + ch * 32, r);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (ch * 32 + i < valid) mx = fmaxf(mx, __uint_as_float(r[i]));
+            }
+            const float m_new = fmaxf(m, mx * c);
+            const float alpha = fast_exp2(m - m_new);
+            if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
+                // rescale the running output in tensor memory (P_t V_{j-1} has completed:
+                // S_t(j) was issued after it and tcgen05.mma executes in issue order)
+#pragma unroll
+                for (int ch = 0; ch < D / 32; ++ch) {
+                    ptx::tmem_ld32(tO + ch * 32, r);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                    ptx::tmem_st32(tO + ch * 32, r);
+                }
+            }
+            l *= alpha;
+            m = m_new;
+            // pass 2: probabilities, written over S as packed bf16 pairs
+            float sum = 0.f;
+#pragma unroll
+            for (int ch = 0; ch < kBN / 32; ++ch) {
+                ptx::tmem_ld32(tS + ch * 32, r);
+                ptx::tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), c, -m));
+                    float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), c, -m));
+                    if (ch * 32 + 2 * i >= valid) p0 = 0.f;
+                    if (ch * 32 + 2 * i + 1 >= valid) p1 = 0.f;
+                    sum += p0 + p1;
+                    pk[i] = pack_bf16x2(p0, p1);
+                }
+                ptx::tmem_st16(tS + ch * 16, pk);
+            }
+            l += sum;
+            ptx::tmem_wait_st();
+            if (valid < kBN) {
+                // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
+                const int iv = 2 * j + 1, sv = iv % kStages;
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                              p.dev_status);
+                if (!ok) break;
+                if (row >= valid) {
+                    uint8_t* vrow = smem_gen + 2 * kTileBytes + sv * kTileBytes + row * 128;
+#pragma unroll
+                    for (int hf = 0; hf < Cfg::kHalves; ++hf)
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            reinterpret_cast<uint4*>(vrow + hf * kHalfBytes)[q] = make_uint4(0, 0, 0, 0);
+                }
+                ptx::fence_proxy_async_smem();
+            }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t]));
+        }
+        // epilogue: O / l -> bf16 -> global (rows past n_q are not written)
+        const int qrow = q0 + t * kBM + row;
+        uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D;
+        if (n_tiles == 0) {
+            if (qrow < nq)
+                for (int q = 0; q < D / 8; ++q) reinterpret_cast<uint4*>(orow)[q] = make_uint4(0, 0, 0, 0);
+        } else if (ok) {
+            ok = wait_bar(ptx::smem_addr(&ctrl->o_done[t]), (n_tiles - 1) & 1, abort_flag,
+                          p.dev_status);
+            if (ok) {
+                ptx::tc_fence_after_sync();
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+                for (int ch = 0; ch < D / 32; ++ch) {
+                    ptx::tmem_ld32(tO + ch * 32, r);
+                    ptx::tmem_wait_ld();
+                    if (qrow < nq) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(r[8 * q + 0]) * inv, __uint_as_float(r[8 * q + 1]) * inv);
+                            o.y = pack_bf16x2(__uint_as_float(r[8 * q + 2]) * inv, __uint_as_float(r[8 * q + 3]) * inv);
+                            o.z = pack_bf16x2(__uint_as_float(r[8 * q + 4]) * inv, __uint_as_float(r[8 * q + 5]) * inv);
+                            o.w = pack_bf16x2(__uint_as_float(r[8 * q + 6]) * inv, __uint_as_float(r[8 * q + 7]) * inv);
+                            reinterpret_cast<uint4*>(orow + ch * 32)[q] = o;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ================= teardown =================
+    if (*abort_flag) {
+        // give copies and MMAs that are still in flight time to land before tensor memory and
+        // shared memory are given back
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 9) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, 512);
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) ==
+                cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    }
+    return fn;
+}
+
+// [B, rows, H, D] bf16 as a 4-D tensor (D, H, rows, B); box = 64 columns x 1 head x 128 rows.
+static bool make_map(CUtensorMap* map, const void* base, int B, int rows, int H, int D) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    if (rows <= 0) rows = 1;     // never loaded from; keeps the encoder happy
+    cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)rows, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2, (cuuint64_t)rows * H * D * 2};
+    cuuint32_t box[4] = {64, 1, (cuuint32_t)kBN, 1};
+    cuuint32_t elem[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+              elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t region_attention_tc_workspace(int, int, int, int, int, int) { return 0; }
+
+template <int D>
+static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int B, cudaStream_t st) {
+    using Cfg = AttnCfg<D>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(region_attention_tc_kernel<D>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Cfg::kSmemBytes) != cudaSuccess)
+            return REGIONE_CUDA_ERROR;
+        configured = true;
+    }
+    dim3 grid((prm.Nq_cap + 2 * kBM - 1) / (2 * kBM), prm.H, B);
+    region_attention_tc_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, st>>>(
+        maps[0], maps[1], maps[2], maps[3], maps[4], prm);
+    return launch_status(cudaGetLastError());
+}
+
+int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const uint16_t* v_fresh,
+                               const uint16_t* k_cache, const uint16_t* v_cache, const int32_t* n_q,
+                               const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap,
+                               int Nf_cap, int Nc_cap, int H, int D, float scale, uint16_t* out,
+                               void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                               cudaStream_t st) {
+    (void)workspace;
+    (void)workspace_bytes;
+    CUtensorMap maps[5];
+    // an absent segment still needs a valid (never dereferenced) base address
+    const void* kf = Nf_cap > 0 ? (const void*)k_fresh : (const void*)q;
+    const void* vf = Nf_cap > 0 ? (const void*)v_fresh : (const void*)q;
+    const void* kc = Nc_cap > 0 ? (const void*)k_cache : (const void*)q;
+    const void* vc = Nc_cap > 0 ? (const void*)v_cache : (const void*)q;
+    if (!make_map(&maps[0], q, B, Nq_cap, H, D) || !make_map(&maps[1], kf, B, Nf_cap, H, D) ||
+        !make_map(&maps[2], vf, B, Nf_cap, H, D) || !make_map(&maps[3], kc, B, Nc_cap, H, D) ||
+        !make_map(&maps[4], vc, B, Nc_cap, H, D))
+        return REGIONE_CUDA_ERROR;
+    AttnParams prm;
+    prm.n_q = n_q; prm.n_fresh = n_fresh; prm.n_cache = n_cache;
+    prm.Nq_cap = Nq_cap; prm.Nf_cap = Nf_cap; prm.Nc_cap = Nc_cap; prm.H = H;
+    prm.scale_log2e = scale * 1.4426950408889634f;
+    prm.out = out; prm.dev_status = dev_status;
+    return D == 64 ? launch_tc<64>(maps, prm, B, st) : launch_tc<128>(maps, prm, B, st);
+}
+
+}  // namespace regione

@@ -1,0 +1,50 @@
+// Shared host/device helpers for the libregione kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "regione.h"
+
+namespace regione {
+
+// Records the first device-side anomaly; later ones do not overwrite it.
+__device__ __forceinline__ void record_status(int32_t* dev_status, int code) {
+    if (dev_status != nullptr) atomicCAS(dev_status, REGIONE_DEV_OK, code);
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Two fp32 -> packed bf16x2 (round to nearest even); `lo` lands in bits [15:0].
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&p);
+}
+
+// 2^x on the special-function unit (flush-to-zero, ~2 ulp); 2^-inf = 0.
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint4 ldg128(const void* p) {
+    return __ldg(reinterpret_cast<const uint4*>(p));
+}
+
+// Streaming 128-bit load for data that is read exactly once (bypasses L1 allocation).
+__device__ __forceinline__ uint4 ld_stream128(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int launch_status(cudaError_t e) { return e == cudaSuccess ? REGIONE_OK : REGIONE_CUDA_ERROR; }
+
+}  // namespace regione

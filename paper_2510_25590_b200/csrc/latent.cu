@@ -1,0 +1,111 @@
+// Elementwise latent updates of the region steps: decayed cached velocity with
+// the Euler update of the edited tokens (Sec. 4, case equation of the AVDCache;
+// Sec. 3, Euler sampler equation) and the merge with one-step-predicted
+// unedited tokens (one-step estimation equation; Algorithm 1).
+//
+// Both are HBM-bound: one thread owns 8 channels (one 128-bit access per
+// tensor), fp32 math, bf16 round-to-nearest-even on the way out.
+#include "common.cuh"
+
+namespace regione {
+
+constexpr int kLatThreads = 256;
+
+__device__ __forceinline__ uint4 axpy8(uint4 x, uint4 v, float a) {   // x + a * v, per bf16 lane
+    uint4 o;
+    o.x = pack_bf16x2(fmaf(a, bf16_lo(v.x), bf16_lo(x.x)), fmaf(a, bf16_hi(v.x), bf16_hi(x.x)));
+    o.y = pack_bf16x2(fmaf(a, bf16_lo(v.y), bf16_lo(x.y)), fmaf(a, bf16_hi(v.y), bf16_hi(x.y)));
+    o.z = pack_bf16x2(fmaf(a, bf16_lo(v.z), bf16_lo(x.z)), fmaf(a, bf16_hi(v.z), bf16_hi(x.z)));
+    o.w = pack_bf16x2(fmaf(a, bf16_lo(v.w), bf16_lo(x.w)), fmaf(a, bf16_hi(v.w), bf16_hi(x.w)));
+    return o;
+}
+
+// x_e <- x_e - dt * (scale * v_in); optionally v_cache_out <- v_in.  One thread = 8 channels.
+__global__ void __launch_bounds__(kLatThreads)
+velocity_decay_kernel(const uint4* __restrict__ v_in, float neg_dt_scale, uint4* __restrict__ x_e,
+                      uint4* __restrict__ v_cache_out, const int32_t* __restrict__ n_edit,
+                      int Ne_cap, int cpr, int32_t* dev_status) {
+    const int b = blockIdx.y;
+    int ne = n_edit[b];
+    if (ne < 0 || ne > Ne_cap) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) record_status(dev_status, REGIONE_DEV_BOUNDS);
+        ne = max(0, min(ne, Ne_cap));
+    }
+    const unsigned live = (unsigned)ne * (unsigned)cpr;
+    const unsigned e = blockIdx.x * (unsigned)kLatThreads + threadIdx.x;
+    if (e >= live) return;
+    const size_t off = (size_t)b * Ne_cap * cpr + e;
+    const uint4 v = ld_stream128(v_in + off);
+    const uint4 x = x_e[off];
+    x_e[off] = axpy8(x, v, neg_dt_scale);
+    if (v_cache_out != nullptr) v_cache_out[off] = v;
+}
+
+// x_out[n] = slot[n] >= 0 ? x_e[slot[n]] : x_full[n] - dt * v_last[n].  One thread = 8 channels.
+__global__ void __launch_bounds__(kLatThreads)
+merge_kernel(const uint4* x_full, const uint4* __restrict__ v_last,
+             const uint4* __restrict__ x_e, const int32_t* __restrict__ slot, float neg_dt, int N,
+             int Ne_cap, int cpr, uint4* x_out, int32_t* dev_status) {
+    const int b = blockIdx.y;
+    const unsigned total = (unsigned)N * (unsigned)cpr;
+    const unsigned e = blockIdx.x * (unsigned)kLatThreads + threadIdx.x;
+    if (e >= total) return;
+    const unsigned n = e / (unsigned)cpr;
+    const unsigned c = e - n * (unsigned)cpr;
+    const int s = slot[(size_t)b * N + n];
+    const size_t off = (size_t)b * N * cpr + e;
+    if (s >= 0) {
+        if (s >= Ne_cap) {
+            record_status(dev_status, REGIONE_DEV_BOUNDS);
+            return;
+        }
+        x_out[off] = ldg128(x_e + ((size_t)b * Ne_cap + s) * cpr + c);
+    } else {
+        const uint4 x = x_full[off];
+        const uint4 v = ld_stream128(v_last + off);
+        x_out[off] = axpy8(x, v, neg_dt);
+    }
+}
+
+}  // namespace regione
+
+using namespace regione;
+
+extern "C" int regione_velocity_decay(const regione_bf16* v_in, float scale, float dt,
+                                      regione_bf16* x_e, regione_bf16* v_cache_out,
+                                      const int32_t* n_edit, int B, int Ne_cap, int C,
+                                      int32_t* dev_status, void* stream) {
+    if (!v_in || !x_e || !n_edit) return REGIONE_INVALID_ARG;
+    if (B < 0 || Ne_cap < 0 || C < 1) return REGIONE_INVALID_ARG;
+    if (!aligned16(v_in) || !aligned16(x_e) || !aligned16(v_cache_out)) return REGIONE_INVALID_ARG;
+    if ((C & 7) != 0 || B > 65535) return REGIONE_UNSUPPORTED;
+    const long long cpr = C / 8, total = (long long)Ne_cap * cpr;
+    if (total + kLatThreads >= 0x7fffffffLL) return REGIONE_UNSUPPORTED;
+    if (B == 0 || Ne_cap == 0) return REGIONE_OK;
+    dim3 grid((unsigned)((total + kLatThreads - 1) / kLatThreads), B);
+    // scale * v is formed first in fp32, then the Euler step: x - dt * (scale * v)
+    velocity_decay_kernel<<<grid, kLatThreads, 0, (cudaStream_t)stream>>>(
+        (const uint4*)v_in, -(dt * scale), (uint4*)x_e, (uint4*)v_cache_out, n_edit, Ne_cap,
+        (int)cpr, dev_status);
+    return launch_status(cudaGetLastError());
+}
+
+extern "C" int regione_merge(const regione_bf16* x_full, const regione_bf16* v_last_full,
+                             const regione_bf16* x_e, const int32_t* slot, float dt_unedited, int B,
+                             int N, int Ne_cap, int C, regione_bf16* x_out, int32_t* dev_status,
+                             void* stream) {
+    if (!x_full || !v_last_full || !slot || !x_out) return REGIONE_INVALID_ARG;
+    if (B < 0 || N < 1 || Ne_cap < 0 || C < 1) return REGIONE_INVALID_ARG;
+    if (Ne_cap > 0 && !x_e) return REGIONE_INVALID_ARG;
+    if (!aligned16(x_full) || !aligned16(v_last_full) || !aligned16(x_e) || !aligned16(x_out))
+        return REGIONE_INVALID_ARG;
+    if ((C & 7) != 0 || B > 65535) return REGIONE_UNSUPPORTED;
+    const long long cpr = C / 8, total = (long long)N * cpr;
+    if (total + kLatThreads >= 0x7fffffffLL) return REGIONE_UNSUPPORTED;
+    if (B == 0) return REGIONE_OK;
+    dim3 grid((unsigned)((total + kLatThreads - 1) / kLatThreads), B);
+    merge_kernel<<<grid, kLatThreads, 0, (cudaStream_t)stream>>>(
+        (const uint4*)x_full, (const uint4*)v_last_full, (const uint4*)x_e, slot, -dt_unedited, N,
+        Ne_cap, (int)cpr, (uint4*)x_out, dev_status);
+    return launch_status(cudaGetLastError());
+}

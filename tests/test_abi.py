@@ -1,0 +1,81 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header declares, validates
+arguments on the host, and its host-only entry points agree with the oracle (CPU only)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import regione_oracle as orc
+from paper_2510_25590_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _header_symbols():
+    text = open(os.path.join(ROOT, "include", "regione.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(regione_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2510_25590_b200 import build
+    build.build()
+    lib = binding.load()
+    names = _header_symbols()
+    assert len(names) >= 12
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(binding.SIGNATURES) == names          # the binding covers exactly the header
+    assert binding.version() >= 100
+    assert binding.status_string(binding.UNSUPPORTED) == "REGIONE_UNSUPPORTED"
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    with pytest.raises(binding.RegionEError):
+        binding.load(str(tmp_path / "nope.so"))
+
+
+def test_argument_validation_happens_on_the_host():
+    lib = binding.load()
+    null = None
+    assert lib.regione_partition(null, null, null, 1, 8, 16, 0.5, 0, 0.9, null, null, null, null, null,
+                                 null, null, null) == binding.INVALID_ARG
+    fake = ctypes.c_void_p(4096)
+    assert lib.regione_partition(fake, fake, fake, 1, 8, 12, 0.5, 0, 0.9, fake, fake, fake, fake, fake,
+                                 null, null, null) == binding.UNSUPPORTED         # C % 8 != 0
+    assert lib.regione_partition(fake, fake, fake, 1, 8, 16, 0.5, 7, 0.9, fake, fake, fake, fake, fake,
+                                 null, null, null) == binding.INVALID_ARG         # unknown metric
+    odd = ctypes.c_void_p(4100)
+    assert lib.regione_gather(odd, fake, fake, 1, 4, 4, 4, 32, fake, null, null) == binding.INVALID_ARG
+    assert lib.regione_gather(fake, fake, fake, 1, 4, 4, 4, 24, fake, null, null) == binding.UNSUPPORTED
+    assert lib.regione_scatter(fake, fake, fake, 1, 8, 4, 8, 32, fake, null, null) == binding.INVALID_ARG
+    assert lib.regione_rikv_store(fake, fake, fake, fake, 1, 8, 8, 3, 3, fake, fake, null, null) \
+        == binding.UNSUPPORTED
+    assert lib.regione_region_attention(fake, fake, fake, fake, fake, fake, fake, fake, 1, 8, 8, 8, 2, 96,
+                                        0.0, fake, null, 0, null, null) == binding.UNSUPPORTED
+    assert lib.regione_region_attention(fake, null, null, fake, fake, fake, fake, fake, 1, 8, 8, 8, 2, 64,
+                                        0.0, fake, null, 0, null, null) == binding.INVALID_ARG
+    assert lib.regione_velocity_decay(fake, 1.0, 0.1, fake, null, fake, 1, 8, 10, null, null) \
+        == binding.UNSUPPORTED
+    assert lib.regione_merge(fake, fake, null, fake, 0.1, 1, 8, 4, 16, fake, null, null) \
+        == binding.INVALID_ARG
+    assert lib.regione_mask_open_close(fake, 1, 200, 200, ctypes.c_void_p(8192), fake, fake, fake, fake,
+                                       null, null) == binding.UNSUPPORTED
+    assert lib.regione_region_attention_workspace(1, 128, 128, 128, 4, 96) == 0
+
+
+def test_avd_step_matches_oracle():
+    T = 28
+    ts = np.arange(T + 1) / T
+    g = 0.9 + 0.1 * np.random.default_rng(5).random(T + 1)
+    for delta in (-1.0, 0.02, 0.04, 0.1, 1.0):
+        p_lib = p_orc = 1.0
+        for j in range(21, 2, -1):
+            dt = ts[j + 1] - ts[j]
+            p_lib, r_lib = binding.avd_step(p_lib, dt, g[j], delta)
+            p_orc, r_orc = orc.avd_step(p_orc, dt, g[j], delta)
+            assert r_lib == r_orc and abs(p_lib - p_orc) < 1e-15
+    with pytest.raises(binding.RegionEError):
+        binding._check(binding.load().regione_avd_step(None, 0.1, 1.0, 0.1, None), "avd")

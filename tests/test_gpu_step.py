@@ -1,0 +1,68 @@
+"""GPU parity: the whole region-aware step (every hot-path stage chained) against the oracle chain."""
+import numpy as np
+import pytest
+
+from gpu_util import assert_close, dev_bf16, host_f64
+from oracle import step_oracle
+from paper_2510_25590_b200 import binding, synth
+from paper_2510_25590_b200.step import RegionStep, StepShapes, plan_capacity
+
+pytestmark = pytest.mark.gpu
+
+
+def run_step(wl, membership="edited_queries", ratio=None):
+    import torch
+    lat = synth.make_latents(wl, ratio)
+    qkv = synth.make_qkv_full(wl)
+    t, scale, dt, dt_u = lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0
+    d = {k: dev_bf16(lat[k]) for k in ("x_t", "v", "ref")}
+    dq, dk, dv = (dev_bf16(qkv[k]) for k in ("q", "k", "v"))
+    metric = binding.METRIC_COSINE if wl.metric == "cosine" else binding.METRIC_L2
+    cap = plan_capacity(d["x_t"], d["v"], d["ref"], t, metric, wl.threshold)
+    shp = StepShapes(wl.batch, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads, wl.head_dim, cap,
+                     metric, wl.threshold,
+                     binding.ROWS_PAPER if membership == "paper" else binding.ROWS_EDITED_QUERIES)
+    step = RegionStep(shp)
+    step.o_full.fill_(0)
+    step.run(d["x_t"], d["v"], d["ref"], dq, dk, dv, t, scale, dt, dt_u)
+    torch.cuda.synchronize()
+    assert int(step.dev_status[0]) == 0
+    want = step_oracle.region_step(wl, lat, qkv, t, np.float32(scale), np.float32(dt), np.float32(dt_u),
+                                   membership)
+    p = want["partition"]
+    assert np.array_equal(step.mask.cpu().numpy(), p["mask"])
+    assert np.array_equal(step.n_edit.cpu().numpy(), p["n_edit"])
+    assert np.array_equal(step.slot.cpu().numpy(), p["slot"])
+    assert np.array_equal(step.n_q.cpu().numpy(), want["n_q"])
+    assert np.array_equal(step.n_cache.cpu().numpy(), want["n_cache"])
+    for b in range(wl.batch):
+        nq, nc = int(want["n_q"][b]), int(want["n_cache"][b])
+        assert np.array_equal(step.query_rows[b, :nq].cpu().numpy(), want["query_rows"][b, :nq])
+        assert np.array_equal(step.cache_rows[b, :nc].cpu().numpy(), want["cache_rows"][b, :nc])
+        assert np.array_equal(host_f64(step.k_cache[b, :nc]), want["k_cache"][b, :nc])      # copies: bit-exact
+        assert np.array_equal(host_f64(step.v_cache[b, :nc]), want["v_cache"][b, :nc])
+        assert_close(host_f64(step.o_e[b, :nq]), want["o_e"][b, :nq], "attention rows")
+        ne = int(p["n_edit"][b])
+        assert_close(host_f64(step.x_e[b, :ne]), want["x_e"][b, :ne], "x_e")
+    assert_close(host_f64(step.o_full), want["o_full"], "scattered attention output")
+    assert_close(host_f64(step.x_out), want["x_out"], "merged latents")
+
+
+def test_config1_whole_step():
+    run_step(synth.WORKLOADS[1])
+
+
+def test_config1_whole_step_paper_membership():
+    run_step(synth.WORKLOADS[1], membership="paper")
+
+
+def test_config5_shape_small_batch_of_four():
+    run_step(synth.scaled_workload(synth.WORKLOADS[5], grid=(24, 24), n_text=48, heads=4))
+
+
+def test_config4_shape_small_l2_metric():
+    run_step(synth.scaled_workload(synth.WORKLOADS[4], grid=(24, 24), n_text=32, heads=4), membership="paper")
+
+
+def test_zero_edit_mask_is_one_step_prediction_everywhere():
+    run_step(synth.scaled_workload(synth.WORKLOADS[2], grid=(16, 16), n_text=16, heads=2), ratio=0.0)
