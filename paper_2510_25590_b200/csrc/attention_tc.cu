@@ -18,6 +18,12 @@
 // softmax and their V rows zeroed in shared memory, so garbage (even NaN)
 // behind the live prefix cannot leak.
 //
+// Occupancy: the key tiles of one (request, head, query pair) can be split over
+// several CTAs (split-KV).  Each split then writes its unnormalised output and
+// its (max, sum) pair to the caller's workspace and a small second kernel
+// merges the splits.  The split count is chosen on the host from the
+// capacities so that the grid fills the SMs.
+//
 // Every wait is bounded: if a barrier does not complete within ~2 s the CTA
 // records REGIONE_DEV_TIMEOUT, all roles leave their loops, tensor memory is
 // released and the kernel ends normally.
@@ -62,6 +68,10 @@ struct AttnParams {
     float scale_log2e;
     uint16_t* out;
     int32_t* dev_status;
+    int n_splits;        // CTAs sharing the key tiles of one (request, head, query pair)
+    int Nq_pad;          // Nq_cap rounded up to a whole query pair (row pitch of the partials)
+    float* part_o;       // [B, n_splits, Nq_pad, H, D] unnormalised outputs (n_splits > 1)
+    float2* part_ml;     // [B, n_splits, Nq_pad, H]    (running max in the exp2 domain, sum)
 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
@@ -79,6 +89,60 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
+// One 128-key tile of the online softmax for one query row (thread = row).  All 128 logits are
+// pulled from tensor memory with one wait, the probabilities go back over S as packed bf16.
+// The reference maximum `m` is only raised (and O rescaled) when a tile maximum exceeds it by
+// more than 2^8: until then probabilities may reach 256, which fp32 sums and bf16 hold fine.
+template <int D, bool MASK>
+__device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int valid, float c,
+                                             bool first, float& m, float& l) {
+    uint32_t s[128];
+    ptx::tmem_ld32(tS, s);
+    ptx::tmem_ld32(tS + 32, s + 32);
+    ptx::tmem_ld32(tS + 64, s + 64);
+    ptx::tmem_ld32(tS + 96, s + 96);
+    ptx::tmem_wait_ld();
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int i = 0; i < 128; ++i) {
+        float v = __uint_as_float(s[i]);
+        if (MASK && i >= valid) v = -INFINITY;
+        mx[i & 3] = fmaxf(mx[i & 3], v);
+    }
+    const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
+    if (first) {
+        m = mt;
+    } else if (__any_sync(0xffffffffu, mt > m + 8.f)) {
+        const float m_new = fmaxf(m, mt);
+        const float alpha = fast_exp2(m - m_new);
+        uint32_t r[32];
+#pragma unroll
+        for (int ch = 0; ch < D / 32; ++ch) {
+            ptx::tmem_ld32(tO + ch * 32, r);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            ptx::tmem_st32(tO + ch * 32, r);
+        }
+        l *= alpha;
+        m = m_new;
+    }
+    float sum[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t pk[64];
+#pragma unroll
+    for (int i = 0; i < 64; ++i) {
+        float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, -m));
+        float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m));
+        if (MASK && 2 * i >= valid) p0 = 0.f;
+        if (MASK && 2 * i + 1 >= valid) p1 = 0.f;
+        sum[i & 3] += p0 + p1;
+        pk[i] = pack_bf16x2(p0, p1);
+    }
+    ptx::tmem_st32(tS, pk);
+    ptx::tmem_st32(tS + 32, pk + 32);
+    l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+}
+
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
@@ -91,7 +155,8 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     constexpr int kTileBytes = Cfg::kTileBytes;
 
     const int b = blockIdx.z, h = blockIdx.y;
-    const int q0 = blockIdx.x * (2 * kBM);
+    const int split = blockIdx.x % p.n_splits;
+    const int q0 = (blockIdx.x / p.n_splits) * (2 * kBM);
     int nq = p.n_q[b], nf = p.n_fresh[b], nc = p.n_cache[b];
     if (nq < 0 || nq > p.Nq_cap || nf < 0 || nf > p.Nf_cap || nc < 0 || nc > p.Nc_cap) {
         if (threadIdx.x == 0) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
@@ -103,7 +168,10 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int ntq = (nq - q0 > kBM) ? 2 : 1;            // live query tiles of this CTA
     const int nt_c = (nc + kBN - 1) / kBN;
     const int nt_f = (nf + kBN - 1) / kBN;
-    const int n_tiles = nt_c + nt_f;
+    const int n_tiles_all = nt_c + nt_f;
+    // this CTA's share of the key tiles: [j_first, j_first + n_tiles)
+    const int j_first = (int)(((long long)split * n_tiles_all) / p.n_splits);
+    const int n_tiles = (int)(((long long)(split + 1) * n_tiles_all) / p.n_splits) - j_first;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -139,7 +207,8 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     const uint32_t tmem = ctrl->tmem_base;
 
     // tile j -> (segment, first row, live rows)
-    auto tile_seg = [&](int j, bool& cached, int& row0, int& valid) {
+    auto tile_seg = [&](int jl, bool& cached, int& row0, int& valid) {
+        const int j = j_first + jl;
         cached = j < nt_c;
         const int jj = cached ? j : j - nt_c;
         row0 = jj * kBN;
@@ -150,8 +219,8 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         // ================= TMA producer =================
         if (lane == 0) {
             ptx::prefetch_tensormap(&tm_q);
-            ptx::prefetch_tensormap(nt_c ? &tm_kc : &tm_kf);
-            ptx::prefetch_tensormap(nt_c ? &tm_vc : &tm_vf);
+            ptx::prefetch_tensormap(j_first < nt_c ? &tm_kc : &tm_kf);
+            ptx::prefetch_tensormap(j_first < nt_c ? &tm_vc : &tm_vf);
             const uint32_t qbar = ptx::smem_addr(&ctrl->q_full);
             ptx::mbar_arrive_expect_tx(qbar, ntq * kTileBytes);
             for (int t = 0; t < ntq; ++t)
@@ -249,58 +318,16 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
-        uint32_t r[32];
         for (int j = 0; j < n_tiles; ++j) {
             ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             bool cached; int row0, valid;
             tile_seg(j, cached, row0, valid);
-            // pass 1: row maximum over the live columns
-            float mx = -INFINITY;
-#pragma unroll
-            for (int ch = 0; ch < kBN / 32; ++ch) {
-                ptx::tmem_ld32(tS + ch * 32, r);
-                ptx::tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (ch * 32 + i < valid) mx = fmaxf(mx, __uint_as_float(r[i]));
-            }
-            const float m_new = fmaxf(m, mx * c);
-            const float alpha = fast_exp2(m - m_new);
-            if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
-                // rescale the running output in tensor memory (P_t V_{j-1} has completed:
-                // S_t(j) was issued after it and tcgen05.mma executes in issue order)
-#pragma unroll
-                for (int ch = 0; ch < D / 32; ++ch) {
-                    ptx::tmem_ld32(tO + ch * 32, r);
-                    ptx::tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                    ptx::tmem_st32(tO + ch * 32, r);
-                }
-            }
-            l *= alpha;
-            m = m_new;
-            // pass 2: probabilities, written over S as packed bf16 pairs
-            float sum = 0.f;
-#pragma unroll
-            for (int ch = 0; ch < kBN / 32; ++ch) {
-                ptx::tmem_ld32(tS + ch * 32, r);
-                ptx::tmem_wait_ld();
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), c, -m));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), c, -m));
-                    if (ch * 32 + 2 * i >= valid) p0 = 0.f;
-                    if (ch * 32 + 2 * i + 1 >= valid) p1 = 0.f;
-                    sum += p0 + p1;
-                    pk[i] = pack_bf16x2(p0, p1);
-                }
-                ptx::tmem_st16(tS + ch * 16, pk);
-            }
-            l += sum;
+            // (P_t V_{j-1} has completed here: S_t(j) was issued after it and tcgen05.mma executes
+            // in issue order, so O_t may be rescaled and P_t overwritten)
+            if (valid == kBN) softmax_tile<D, false>(tS, tO, valid, c, j == 0, m, l);
+            else softmax_tile<D, true>(tS, tO, valid, c, j == 0, m, l);
             ptx::tmem_wait_st();
             if (valid < kBN) {
                 // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
@@ -321,23 +348,29 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t]));
         }
-        // epilogue: O / l -> bf16 -> global (rows past n_q are not written)
+        // epilogue (rows past n_q are not written)
         const int qrow = q0 + t * kBM + row;
-        uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D;
-        if (n_tiles == 0) {
-            if (qrow < nq)
-                for (int q = 0; q < D / 8; ++q) reinterpret_cast<uint4*>(orow)[q] = make_uint4(0, 0, 0, 0);
-        } else if (ok) {
+        const bool live = qrow < nq;
+        if (n_tiles > 0 && ok) {
             ok = wait_bar(ptx::smem_addr(&ctrl->o_done[t]), (n_tiles - 1) & 1, abort_flag,
                           p.dev_status);
-            if (ok) {
-                ptx::tc_fence_after_sync();
+            if (ok) ptx::tc_fence_after_sync();
+        }
+        if (p.n_splits == 1) {
+            // O / l -> bf16 -> out
+            uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D;
+            if (n_tiles == 0) {
+                if (live)
+                    for (int q = 0; q < D / 8; ++q)
+                        reinterpret_cast<uint4*>(orow)[q] = make_uint4(0, 0, 0, 0);
+            } else if (ok) {
                 const float inv = l > 0.f ? 1.f / l : 0.f;
+                uint32_t r[32];
 #pragma unroll
                 for (int ch = 0; ch < D / 32; ++ch) {
                     ptx::tmem_ld32(tO + ch * 32, r);
                     ptx::tmem_wait_ld();
-                    if (qrow < nq) {
+                    if (live) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             uint4 o;
@@ -349,6 +382,27 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                         }
                     }
                 }
+            }
+        } else {
+            // unnormalised O and (m, l) of this split -> workspace; a split without keys has l = 0
+            const size_t prow = (((size_t)b * p.n_splits + split) * p.Nq_pad + qrow) * p.H + h;
+            if (n_tiles == 0) {
+                if (live) p.part_ml[prow] = make_float2(-INFINITY, 0.f);
+            } else if (ok) {
+                float* po = p.part_o + prow * D;
+                uint32_t r[32];
+#pragma unroll
+                for (int ch = 0; ch < D / 32; ++ch) {
+                    ptx::tmem_ld32(tO + ch * 32, r);
+                    ptx::tmem_wait_ld();
+                    if (live) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            reinterpret_cast<uint4*>(po + ch * 32)[q] =
+                                make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                    }
+                }
+                if (live) p.part_ml[prow] = make_float2(m, l);
             }
         }
     }
@@ -368,7 +422,80 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
 }
 
+// Merges the splits of one output row: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
+// One warp per (request, query row, head); a lane owns D / 32 consecutive columns.
+template <int D>
+__global__ void __launch_bounds__(256)
+region_attention_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml,
+                                const int32_t* __restrict__ n_q, int Nq_cap, int Nq_pad, int H,
+                                int n_splits, uint16_t* __restrict__ out) {
+    const int b = blockIdx.z;
+    const int lane = threadIdx.x & 31;
+    const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);     // (row, head) pair
+    const int qrow = (int)(w / H), h = (int)(w % H);
+    const int nq = max(0, min(n_q[b], Nq_cap));
+    if (qrow >= nq) return;
+    constexpr int E = D / 32;
+    float M = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) {
+        const float2 ml = part_ml[(((size_t)b * n_splits + s) * Nq_pad + qrow) * H + h];
+        if (ml.y > 0.f) M = fmaxf(M, ml.x);
+    }
+    float acc[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    float L = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const size_t prow = (((size_t)b * n_splits + s) * Nq_pad + qrow) * H + h;
+        const float2 ml = part_ml[prow];
+        if (!(ml.y > 0.f)) continue;
+        const float wgt = fast_exp2(ml.x - M);
+        L = fmaf(wgt, ml.y, L);
+        const float* po = part_o + prow * D + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = fmaf(wgt, po[e], acc[e]);
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    uint16_t* orow = out + (((size_t)b * Nq_cap + qrow) * H + h) * D + lane * E;
+#pragma unroll
+    for (int e = 0; e < E; e += 2)
+        *reinterpret_cast<uint32_t*>(orow + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
+}
+
 // ---- host side ---------------------------------------------------------------------------------
+
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            return 148;
+    }
+    return n;
+}
+
+// Split count from the capacities alone (so the workspace query and the launch agree): the
+// smallest count, at most 8 and leaving at least 4 key tiles per split, whose grid wastes the
+// least of its last wave.
+static int choose_splits(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H) {
+    const long long items = (long long)((Nq_cap + 2 * kBM - 1) / (2 * kBM)) * H * B;
+    const int tiles = (Nf_cap + kBN - 1) / kBN + (Nc_cap + kBN - 1) / kBN;
+    const int sms = sm_count();
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= 8 && (s == 1 || tiles / s >= 4); ++s) {
+        const long long ctas = items * s;
+        const double eff = (double)ctas / (double)(((ctas + sms - 1) / sms) * sms);
+        if (eff > best_eff + 0.02) {
+            best_eff = eff;
+            best = s;
+        }
+    }
+    return best;
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -403,7 +530,14 @@ static bool make_map(CUtensorMap* map, const void* base, int B, int rows, int H,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-size_t region_attention_tc_workspace(int, int, int, int, int, int) { return 0; }
+static inline int pad_rows(int Nq_cap) { return (Nq_cap + 2 * kBM - 1) / (2 * kBM) * (2 * kBM); }
+
+size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D) {
+    const int s = choose_splits(B, Nq_cap, Nf_cap, Nc_cap, H);
+    if (s == 1) return 0;
+    const size_t rows = (size_t)B * s * pad_rows(Nq_cap) * H;
+    return ((rows * D * sizeof(float) + 255) & ~(size_t)255) + rows * sizeof(float2);
+}
 
 template <int D>
 static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int B, cudaStream_t st) {
@@ -416,9 +550,16 @@ static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int B, cuda
             return REGIONE_CUDA_ERROR;
         configured = true;
     }
-    dim3 grid((prm.Nq_cap + 2 * kBM - 1) / (2 * kBM), prm.H, B);
+    dim3 grid((prm.Nq_cap + 2 * kBM - 1) / (2 * kBM) * prm.n_splits, prm.H, B);
     region_attention_tc_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, st>>>(
         maps[0], maps[1], maps[2], maps[3], maps[4], prm);
+    if (cudaGetLastError() != cudaSuccess) return REGIONE_CUDA_ERROR;
+    if (prm.n_splits > 1) {
+        const long long warps = (long long)prm.Nq_cap * prm.H;
+        dim3 cgrid((unsigned)((warps + 7) / 8), 1, B);
+        region_attention_combine_kernel<D><<<cgrid, 256, 0, st>>>(
+            prm.part_o, prm.part_ml, prm.n_q, prm.Nq_cap, prm.Nq_pad, prm.H, prm.n_splits, prm.out);
+    }
     return launch_status(cudaGetLastError());
 }
 
@@ -428,7 +569,6 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
                                int Nf_cap, int Nc_cap, int H, int D, float scale, uint16_t* out,
                                void* workspace, size_t workspace_bytes, int32_t* dev_status,
                                cudaStream_t st) {
-    (void)workspace;
     (void)workspace_bytes;
     CUtensorMap maps[5];
     // an absent segment still needs a valid (never dereferenced) base address
@@ -445,6 +585,15 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
     prm.Nq_cap = Nq_cap; prm.Nf_cap = Nf_cap; prm.Nc_cap = Nc_cap; prm.H = H;
     prm.scale_log2e = scale * 1.4426950408889634f;
     prm.out = out; prm.dev_status = dev_status;
+    prm.n_splits = choose_splits(B, Nq_cap, Nf_cap, Nc_cap, H);
+    prm.Nq_pad = pad_rows(Nq_cap);
+    prm.part_o = nullptr; prm.part_ml = nullptr;
+    if (prm.n_splits > 1) {
+        const size_t rows = (size_t)B * prm.n_splits * prm.Nq_pad * H;
+        prm.part_o = reinterpret_cast<float*>(workspace);
+        prm.part_ml = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(workspace) +
+                                                ((rows * D * sizeof(float) + 255) & ~(size_t)255));
+    }
     return D == 64 ? launch_tc<64>(maps, prm, B, st) : launch_tc<128>(maps, prm, B, st);
 }
 
