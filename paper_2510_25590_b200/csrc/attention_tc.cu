@@ -191,7 +191,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
         for (int t = 0; t < 2; ++t) {
             ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t]), kBM);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t]), kBM / 32);
             ptx::mbar_init(ptx::smem_addr(&ctrl->o_done[t]), 1);
         }
         ctrl->abort_flag = 0;
@@ -247,65 +247,76 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
     } else if (warp == 9) {
         // ================= MMA issuer =================
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
-            constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
-            // S_t = Q_t K^T : both operands K-major, 128-byte swizzle, 8-row groups 1024 B apart.
-            auto issue_s = [&](int t, int stage) {
+        // The whole warp walks the loop and waits on the barriers; one elected lane issues.
+        constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
+        constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
+        constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
+        // K-major operands (Q, K): 128-byte swizzle, LBO unused; V is MN-major: 64-column boxes
+        // kHalfBytes apart (LBO), 8-key groups 1024 B apart (SBO).
+        const uint32_t q_lo = ptx::smem_desc_lo(sQ, 16);
+        const uint32_t k_lo = ptx::smem_desc_lo(sKV, 16);
+        const uint32_t v_lo = ptx::smem_desc_lo(sKV, kHalfBytes);
+        // S_t = Q_t K^T
+        auto issue_s = [&](int t, int stage) {
+            const uint32_t a0 = q_lo + ((t * kTileBytes) >> 4);
+            const uint32_t b0 = k_lo + ((stage * kTileBytes) >> 4);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                    const uint64_t da = ptx::smem_desc_sw128(sQ + t * kTileBytes + off, 16, 1024);
-                    const uint64_t db = ptx::smem_desc_sw128(sKV + stage * kTileBytes + off, 16, 1024);
-                    ptx::mma_ss(tmem + t * kBN, da, db, idesc_s, kk > 0);
-                }
-            };
-            // O_t (+)= P_t V : A from tensor memory (bf16 pairs, 8 columns per 16 keys), B = V
-            // MN-major: 64-column boxes 16 KB apart (LBO), 8-key groups 1024 B apart (SBO).
-            auto issue_pv = [&](int t, int stage, bool accumulate) {
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                ptx::mma_ss(tmem + t * kBN, ptx::smem_desc_join(a0 + off, hi_k),
+                            ptx::smem_desc_join(b0 + off, hi_k), idesc_s, kk > 0);
+            }
+        };
+        // O_t (+)= P_t V : A from tensor memory (bf16 pairs, 8 columns per 16 keys)
+        auto issue_pv = [&](int t, int stage, bool accumulate) {
+            const uint32_t b0 = v_lo + ((stage * kTileBytes) >> 4);
 #pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk) {
-                    const uint64_t db =
-                        ptx::smem_desc_sw128(sKV + stage * kTileBytes + kk * 2048, kHalfBytes, 1024);
-                    ptx::mma_ts(tmem + 256 + t * D, tmem + t * kBN + kk * 8, db, idesc_pv,
-                                (accumulate || kk > 0) ? 1u : 0u);
-                }
-            };
-            bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
-            if (ok && n_tiles > 0) {
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[0]), 0, abort_flag, p.dev_status);
-                if (ok) {
-                    ptx::tc_fence_after_sync();
+            for (int kk = 0; kk < kBN / 16; ++kk)
+                ptx::mma_ts(tmem + 256 + t * D, tmem + t * kBN + kk * 8,
+                            ptx::smem_desc_join(b0 + ((kk * 2048) >> 4), hi_k), idesc_pv,
+                            (accumulate || kk > 0) ? 1u : 0u);
+        };
+        bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
+        if (ok && n_tiles > 0) {
+            ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[0]), 0, abort_flag, p.dev_status);
+            if (ok) {
+                ptx::tc_fence_after_sync();
+                if (ptx::elect_one()) {
                     for (int t = 0; t < ntq; ++t) {
                         issue_s(t, 0);
                         ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
                     }
                     ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[0]));
                 }
+                __syncwarp();
             }
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int iv = 2 * j + 1, ik = 2 * j + 2;
-                const int sv = iv % kStages, sk = ik % kStages;
-                const bool more = (j + 1 < n_tiles);
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
-                              p.dev_status);
-                for (int t = 0; t < ntq && ok; ++t) {
-                    ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t]), j & 1, abort_flag, p.dev_status);
+        }
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int iv = 2 * j + 1, ik = 2 * j + 2;
+            const int sv = iv % kStages, sk = ik % kStages;
+            const bool more = (j + 1 < n_tiles);
+            ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                          p.dev_status);
+            for (int t = 0; t < ntq && ok; ++t) {
+                ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t]), j & 1, abort_flag, p.dev_status);
+                if (!ok) break;
+                if (more && t == 0) {
+                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / kStages) & 1,
+                                  abort_flag, p.dev_status);
                     if (!ok) break;
-                    ptx::tc_fence_after_sync();
+                }
+                ptx::tc_fence_after_sync();
+                if (ptx::elect_one()) {
                     issue_pv(t, sv, j > 0);
                     ptx::mma_commit(ptx::smem_addr(&ctrl->o_done[t]));
                     if (t == ntq - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sv]));
                     if (more) {
-                        if (t == 0)
-                            ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / kStages) & 1,
-                                          abort_flag, p.dev_status);
-                        if (!ok) break;
                         issue_s(t, sk);
                         ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
                         if (t == ntq - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk]));
                     }
                 }
+                __syncwarp();
             }
         }
     } else if (warp < 4 * ntq) {
@@ -346,7 +357,8 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                 ptx::fence_proxy_async_smem();
             }
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t]));
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t]));
         }
         // epilogue (rows past n_q are not written)
         const int qrow = q0 + t * kBM + row;
