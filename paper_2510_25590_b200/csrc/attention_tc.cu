@@ -6,17 +6,27 @@
 // One CTA = one (request, head, pair of 128-row query tiles).  Warp roles:
 //   warps 0-3  softmax / correction / epilogue of query tile 0 (thread = row)
 //   warps 4-7  the same for query tile 1
-//   warp  8    TMA producer: Q once, then K_j, V_j tiles through a ring of
-//              shared-memory stages; the cached segment and the fresh segment
+//   warp  8    TMA producer: Q once, then K_j, V_j tiles (128 keys) through a ring
+//              of shared-memory stages; the cached segment and the fresh segment
 //              are two tensor maps walked one after the other
-//   warp  9    tcgen05.mma issuer and owner of the tensor-memory allocation
-// Tensor memory (512 columns): S0 | S1 | O0 | O1.  S_t = Q_t K_j^T (fp32) is
-// read back by the softmax warps, the probabilities are written over it as
-// bf16 (P aliases S) and feed O_t += P_t V_j straight from tensor memory.
+//   warps 9,10 tcgen05.mma issuers, one per query tile (the whole warp walks the
+//              loop, one elected lane issues); warp 9 owns the tensor-memory allocation
+//
+// Tensor memory (512 columns): S0a S0b | S1a S1b | O0 | O1.  The logits of a
+// query tile are produced 64 keys at a time, S_t(h) = Q_t K_h^T (fp32, 64
+// columns), alternating between the tile's two buffers a / b.  The softmax
+// warps read S_t(h) back, write the probabilities over it as packed bf16 (P
+// aliases the first 32 columns of its S buffer) and O_t += P_t(h) V_h runs
+// straight from tensor memory.  Because S_t(h+1) sits in the other buffer and
+// is issued before P_t(h) exists, a softmax warp never waits for its own
+// P*V product: the chain S -> softmax -> P*V -> next S of the one-buffer
+// scheme is cut, and the special-function unit (exp2) stays busy.
+//
 // Online softmax in the exp2 domain; O is rescaled in tensor memory only when
-// a row maximum grows.  Rows past a segment's live count are masked in the
-// softmax and their V rows zeroed in shared memory, so garbage (even NaN)
-// behind the live prefix cannot leak.
+// a row maximum grows by more than 2^8 (after waiting for the P*V products
+// already issued for that tile).  Keys past a segment's live count are masked
+// in the softmax and their V rows zeroed in shared memory, so garbage (even
+// NaN) behind the live prefix cannot leak.
 //
 // Occupancy: the key tiles of one (request, head, query pair) can be split over
 // several CTAs (split-KV).  Each split then writes its unnormalised output and
@@ -34,9 +44,10 @@
 
 namespace regione {
 
-constexpr int kAttnThreads = 320;
+constexpr int kAttnThreads = 352;
 constexpr int kBM = 128;                 // query rows per tile
-constexpr int kBN = 128;                 // key rows per tile
+constexpr int kBN = 128;                 // key rows per shared-memory tile
+constexpr int kBH = 64;                  // key rows per S buffer (half a tile)
 constexpr int kHalfBytes = 128 * 64 * 2; // one 128-row x 64-column bf16 box (128-byte rows)
 constexpr long long kTimeoutCycles = 4000000000LL;
 
@@ -53,9 +64,10 @@ struct AttnCtrl {
     uint64_t q_full;
     uint64_t kv_full[6];
     uint64_t kv_empty[6];
-    uint64_t s_full[2];
-    uint64_t p_full[2];
-    uint64_t o_done[2];
+    uint64_t s_full[2][2];      // [query tile][S buffer]
+    uint64_t p_full[2][2];
+    uint64_t o_done[2];         // one completion per P*V product of the tile
+    uint64_t o_final[2];        // completes once, after the tile's last P*V product
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -89,48 +101,30 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
-// One 128-key tile of the online softmax for one query row (thread = row).  All 128 logits are
-// pulled from tensor memory with one wait, the probabilities go back over S as packed bf16.
-// The reference maximum `m` is only raised (and O rescaled) when a tile maximum exceeds it by
-// more than 2^8: until then probabilities may reach 256, which fp32 sums and bf16 hold fine.
-template <int D, bool MASK>
-__device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int valid, float c,
-                                             bool first, float& m, float& l) {
-    uint32_t s[128];
+// Row maximum (times the scale, exp2 domain) of the 64 logits of one S buffer; `s` keeps them.
+template <bool MASK>
+__device__ __forceinline__ float load_logits_max(uint32_t tS, int valid, float c, uint32_t (&s)[kBH]) {
     ptx::tmem_ld32(tS, s);
     ptx::tmem_ld32(tS + 32, s + 32);
-    ptx::tmem_ld32(tS + 64, s + 64);
-    ptx::tmem_ld32(tS + 96, s + 96);
     ptx::tmem_wait_ld();
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-    for (int i = 0; i < 128; ++i) {
+    for (int i = 0; i < kBH; ++i) {
         float v = __uint_as_float(s[i]);
         if (MASK && i >= valid) v = -INFINITY;
         mx[i & 3] = fmaxf(mx[i & 3], v);
     }
-    const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
-    if (first) {
-        m = mt;
-    } else if (__any_sync(0xffffffffu, mt > m + 8.f)) {
-        const float m_new = fmaxf(m, mt);
-        const float alpha = fast_exp2(m - m_new);
-        uint32_t r[32];
-#pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) {
-            ptx::tmem_ld32(tO + ch * 32, r);
-            ptx::tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-            ptx::tmem_st32(tO + ch * 32, r);
-        }
-        l *= alpha;
-        m = m_new;
-    }
+    return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
+}
+
+// p = 2^(s*c - m) for the 64 logits, written over S as packed bf16; returns their fp32 sum.
+template <bool MASK>
+__device__ __forceinline__ float store_probabilities(uint32_t tS, int valid, float c, float m,
+                                                     const uint32_t (&s)[kBH]) {
     float sum[4] = {0.f, 0.f, 0.f, 0.f};
-    uint32_t pk[64];
+    uint32_t pk[kBH / 2];
 #pragma unroll
-    for (int i = 0; i < 64; ++i) {
+    for (int i = 0; i < kBH / 2; ++i) {
         float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, -m));
         float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m));
         if (MASK && 2 * i >= valid) p0 = 0.f;
@@ -139,8 +133,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int valid
         pk[i] = pack_bf16x2(p0, p1);
     }
     ptx::tmem_st32(tS, pk);
-    ptx::tmem_st32(tS + 32, pk + 32);
-    l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+    return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
 template <int D>
@@ -187,12 +180,15 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         ptx::mbar_init(ptx::smem_addr(&ctrl->q_full), 1);
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctrl->kv_full[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_empty[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_empty[s]), ntq);    // one commit per issuer
         }
         for (int t = 0; t < 2; ++t) {
-            ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t]), kBM / 32);
+            for (int u = 0; u < 2; ++u) {
+                ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t][u]), 1);
+                ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t][u]), kBM / 32);
+            }
             ptx::mbar_init(ptx::smem_addr(&ctrl->o_done[t]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->o_final[t]), 1);
         }
         ctrl->abort_flag = 0;
         ptx::fence_barrier_init();
@@ -206,13 +202,19 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     ptx::tc_fence_after_sync();
     const uint32_t tmem = ctrl->tmem_base;
 
-    // tile j -> (segment, first row, live rows)
+    // key tile jl of this CTA -> (segment, first row, live rows); a tile yields one S half when
+    // at most 64 of its keys are live, else two
     auto tile_seg = [&](int jl, bool& cached, int& row0, int& valid) {
         const int j = j_first + jl;
         cached = j < nt_c;
         const int jj = cached ? j : j - nt_c;
         row0 = jj * kBN;
         valid = min(kBN, (cached ? nc : nf) - row0);
+    };
+    auto tile_halves = [&](int jl) {
+        bool cached; int row0, valid;
+        tile_seg(jl, cached, row0, valid);
+        return valid > kBH ? 2 : 1;
     };
 
     if (warp == 8) {
@@ -245,78 +247,104 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                                      row0, b);
             }
         }
-    } else if (warp == 9) {
-        // ================= MMA issuer =================
-        // The whole warp walks the loop and waits on the barriers; one elected lane issues.
-        constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
-        constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
-        constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
-        // K-major operands (Q, K): 128-byte swizzle, LBO unused; V is MN-major: 64-column boxes
-        // kHalfBytes apart (LBO), 8-key groups 1024 B apart (SBO).
-        const uint32_t q_lo = ptx::smem_desc_lo(sQ, 16);
-        const uint32_t k_lo = ptx::smem_desc_lo(sKV, 16);
-        const uint32_t v_lo = ptx::smem_desc_lo(sKV, kHalfBytes);
-        // S_t = Q_t K^T
-        auto issue_s = [&](int t, int stage) {
-            const uint32_t a0 = q_lo + ((t * kTileBytes) >> 4);
-            const uint32_t b0 = k_lo + ((stage * kTileBytes) >> 4);
+    } else if (warp == 9 || warp == 10) {
+        // ================= MMA issuers: warp 9 for query tile 0, warp 10 for query tile 1 ========
+        // Each whole warp walks its loop and waits on the barriers; one elected lane issues.  Two
+        // independent issuers keep the tensor pipe fed: while one sits in the fixed latency of a
+        // barrier wait or a commit, the products of the other execute.
+        const int t = warp - 9;
+        if (t < ntq) {
+            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBH, false);
+            constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
+            constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
+            // K-major operands (Q, K): 128-byte swizzle, LBO unused; V is MN-major: 64-column
+            // boxes kHalfBytes apart (LBO), 8-key groups 1024 B apart (SBO).
+            const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
+            const uint32_t k_lo = ptx::smem_desc_lo(sKV, 16);
+            const uint32_t v_lo = ptx::smem_desc_lo(sKV, kHalfBytes);
+            const uint32_t tS0 = tmem + t * kBN, tOt = tmem + 256 + t * D;
+            // S_t(buffer u) = Q_t K[64 hh .. 64 hh + 64)^T
+            auto issue_s = [&](int stage, int hh, int u) {
+                const uint32_t b0 = k_lo + ((stage * kTileBytes + hh * (kBH * 128)) >> 4);
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
-                ptx::mma_ss(tmem + t * kBN, ptx::smem_desc_join(a0 + off, hi_k),
-                            ptx::smem_desc_join(b0 + off, hi_k), idesc_s, kk > 0);
-            }
-        };
-        // O_t (+)= P_t V : A from tensor memory (bf16 pairs, 8 columns per 16 keys)
-        auto issue_pv = [&](int t, int stage, bool accumulate) {
-            const uint32_t b0 = v_lo + ((stage * kTileBytes) >> 4);
-#pragma unroll
-            for (int kk = 0; kk < kBN / 16; ++kk)
-                ptx::mma_ts(tmem + 256 + t * D, tmem + t * kBN + kk * 8,
-                            ptx::smem_desc_join(b0 + ((kk * 2048) >> 4), hi_k), idesc_pv,
-                            (accumulate || kk > 0) ? 1u : 0u);
-        };
-        bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
-        if (ok && n_tiles > 0) {
-            ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[0]), 0, abort_flag, p.dev_status);
-            if (ok) {
-                ptx::tc_fence_after_sync();
-                if (ptx::elect_one()) {
-                    for (int t = 0; t < ntq; ++t) {
-                        issue_s(t, 0);
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
-                    }
-                    ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[0]));
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                    ptx::mma_ss(tS0 + u * kBH, ptx::smem_desc_join(q_lo + off, hi_k),
+                                ptx::smem_desc_join(b0 + off, hi_k), idesc_s, kk > 0);
                 }
-                __syncwarp();
-            }
-        }
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            const int iv = 2 * j + 1, ik = 2 * j + 2;
-            const int sv = iv % kStages, sk = ik % kStages;
-            const bool more = (j + 1 < n_tiles);
-            ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
-                          p.dev_status);
-            for (int t = 0; t < ntq && ok; ++t) {
-                ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t]), j & 1, abort_flag, p.dev_status);
+            };
+            // O_t (+)= P_t(buffer u) V[64 hh .. 64 hh + 64) : A from tensor memory (bf16 pairs,
+            // 8 columns per 16 keys)
+            auto issue_pv = [&](int stage, int hh, int u, bool accumulate) {
+                const uint32_t b0 = v_lo + ((stage * kTileBytes + hh * (kBH / 16) * 2048) >> 4);
+#pragma unroll
+                for (int kk = 0; kk < kBH / 16; ++kk)
+                    ptx::mma_ts(tOt, tS0 + u * kBH + kk * 8,
+                                ptx::smem_desc_join(b0 + ((kk * 2048) >> 4), hi_k), idesc_pv,
+                                (accumulate || kk > 0) ? 1u : 0u);
+            };
+            // cursor of the next S half to issue: key tile sj, half shh
+            int sj = 0, shh = 0;
+            int s_halves = n_tiles > 0 ? tile_halves(0) : 0;
+            auto s_stage = [&]() { return (2 * sj) % kStages; };
+            auto s_parity = [&]() { return ((2 * sj) / kStages) & 1; };
+            auto s_advance = [&]() {
+                if (++shh == s_halves) {
+                    shh = 0;
+                    ++sj;
+                    s_halves = sj < n_tiles ? tile_halves(sj) : 0;
+                }
+            };
+            bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
+            // prologue: the first two S halves
+            for (int pre = 0; pre < 2 && ok && sj < n_tiles; ++pre) {
+                if (shh == 0)
+                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[s_stage()]), s_parity(), abort_flag,
+                                  p.dev_status);
                 if (!ok) break;
-                if (more && t == 0) {
-                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / kStages) & 1,
-                                  abort_flag, p.dev_status);
-                    if (!ok) break;
-                }
                 ptx::tc_fence_after_sync();
                 if (ptx::elect_one()) {
-                    issue_pv(t, sv, j > 0);
-                    ptx::mma_commit(ptx::smem_addr(&ctrl->o_done[t]));
-                    if (t == ntq - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sv]));
-                    if (more) {
-                        issue_s(t, sk);
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
-                        if (t == ntq - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk]));
-                    }
+                    issue_s(s_stage(), shh, pre);
+                    ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t][pre]));
+                    if (shh == s_halves - 1)
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[s_stage()]));
                 }
                 __syncwarp();
+                s_advance();
+            }
+            int ph = 0;                                     // running index of the P*V half
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int iv = 2 * j + 1, sv = iv % kStages;
+                const int halves = tile_halves(j);
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                              p.dev_status);
+                for (int hh = 0; hh < halves && ok; ++hh, ++ph) {
+                    const int u = ph & 1;
+                    const bool more = sj < n_tiles;         // S half ph + 2 exists
+                    if (more && shh == 0)
+                        ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[s_stage()]), s_parity(),
+                                      abort_flag, p.dev_status);
+                    if (ok)
+                        ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][u]), (ph >> 1) & 1, abort_flag,
+                                      p.dev_status);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    if (ptx::elect_one()) {
+                        issue_pv(sv, hh, u, ph > 0);
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->o_done[t]));
+                        if (j == n_tiles - 1 && hh == halves - 1)
+                            ptx::mma_commit(ptx::smem_addr(&ctrl->o_final[t]));
+                        if (hh == halves - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sv]));
+                        if (more) {
+                            issue_s(s_stage(), shh, u);
+                            ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t][u]));
+                            if (shh == s_halves - 1)
+                                ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[s_stage()]));
+                        }
+                    }
+                    __syncwarp();
+                    if (more) s_advance();
+                }
             }
         }
     } else if (warp < 4 * ntq) {
@@ -324,48 +352,83 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         const int t = warp >> 2;
         const int row = ((warp & 3) << 5) + lane;                  // row of the query tile
         const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
-        const uint32_t tS = tmem + lane_sel + t * kBN;
+        const uint32_t tSt = tmem + lane_sel + t * kBN;
         const uint32_t tO = tmem + lane_sel + 256 + t * D;
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_tiles; ++j) {
-            ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status);
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
+        int ph = 0;                                                // running half index
+        for (int j = 0; j < n_tiles && ok; ++j) {
             bool cached; int row0, valid;
             tile_seg(j, cached, row0, valid);
-            // (P_t V_{j-1} has completed here: S_t(j) was issued after it and tcgen05.mma executes
-            // in issue order, so O_t may be rescaled and P_t overwritten)
-            if (valid == kBN) softmax_tile<D, false>(tS, tO, valid, c, j == 0, m, l);
-            else softmax_tile<D, true>(tS, tO, valid, c, j == 0, m, l);
-            ptx::tmem_wait_st();
-            if (valid < kBN) {
-                // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
-                const int iv = 2 * j + 1, sv = iv % kStages;
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+            const int halves = valid > kBH ? 2 : 1;
+            for (int hh = 0; hh < halves; ++hh, ++ph) {
+                const int u = ph & 1;
+                const uint32_t tS = tSt + u * kBH;
+                ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t][u]), (ph >> 1) & 1, abort_flag,
                               p.dev_status);
                 if (!ok) break;
-                if (row >= valid) {
-                    uint8_t* vrow = smem_gen + 2 * kTileBytes + sv * kTileBytes + row * 128;
+                ptx::tc_fence_after_sync();
+                const int vh = min(kBH, valid - hh * kBH);         // live keys of this half (>= 1)
+                uint32_t s[kBH];
+                const float mt = (vh == kBH) ? load_logits_max<false>(tS, vh, c, s)
+                                             : load_logits_max<true>(tS, vh, c, s);
+                if (ph == 0) {
+                    m = mt;
+                } else if (__any_sync(0xffffffffu, mt > m + 8.f)) {
+                    // raise the reference maximum: every P*V product issued so far for this tile
+                    // (halves 0 .. ph-1) must have landed in O before O is rescaled
+                    ok = wait_bar(ptx::smem_addr(&ctrl->o_done[t]), (ph - 1) & 1, abort_flag,
+                                  p.dev_status);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const float m_new = fmaxf(m, mt);
+                    const float alpha = fast_exp2(m - m_new);
+                    uint32_t r[32];
 #pragma unroll
-                    for (int hf = 0; hf < Cfg::kHalves; ++hf)
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        ptx::tmem_ld32(tO + ch * 32, r);
+                        ptx::tmem_wait_ld();
 #pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            reinterpret_cast<uint4*>(vrow + hf * kHalfBytes)[q] = make_uint4(0, 0, 0, 0);
+                        for (int i = 0; i < 32; ++i)
+                            r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        ptx::tmem_st32(tO + ch * 32, r);
+                    }
+                    l *= alpha;
+                    m = m_new;
                 }
-                ptx::fence_proxy_async_smem();
+                l += (vh == kBH) ? store_probabilities<false>(tS, vh, c, m, s)
+                                 : store_probabilities<true>(tS, vh, c, m, s);
+                ptx::tmem_wait_st();
+                if (hh == 0 && valid < kBN) {
+                    // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
+                    const int iv = 2 * j + 1, sv = iv % kStages;
+                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                                  p.dev_status);
+                    if (!ok) break;
+                    if (row >= valid) {
+                        uint8_t* vrow = smem_gen + 2 * kTileBytes + sv * kTileBytes + row * 128;
+#pragma unroll
+                        for (int hf = 0; hf < Cfg::kHalves; ++hf)
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                reinterpret_cast<uint4*>(vrow + hf * kHalfBytes)[q] = make_uint4(0, 0, 0, 0);
+                    }
+                    ptx::fence_proxy_async_smem();
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t][u]));
             }
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t]));
         }
+        const int n_halves = ph;
         // epilogue (rows past n_q are not written)
         const int qrow = q0 + t * kBM + row;
         const bool live = qrow < nq;
-        if (n_tiles > 0 && ok) {
-            ok = wait_bar(ptx::smem_addr(&ctrl->o_done[t]), (n_tiles - 1) & 1, abort_flag,
-                          p.dev_status);
+        if (n_halves > 0 && ok) {
+            // (o_done advances one phase per product and can be one or two phases short of the
+            // end here, which a parity wait cannot tell apart: hence the barrier of its own)
+            ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status);
             if (ok) ptx::tc_fence_after_sync();
         }
         if (p.n_splits == 1) {
