@@ -68,6 +68,7 @@ struct AttnCtrl {
     uint64_t p_full[2][2];
     uint64_t o_done[2];         // one completion per P*V product of the tile
     uint64_t o_final[2];        // completes once, after the tile's last P*V product
+    uint64_t turn[2];           // turn[t]: the other tile is half way through its exponentials
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -118,9 +119,14 @@ __device__ __forceinline__ float load_logits_max(uint32_t tS, int valid, float c
 }
 
 // p = 2^(s*c - m) for the 64 logits, written over S as packed bf16; returns their fp32 sum.
+// After the first half of the exponentials lane 0 arrives on `turn_bar` (if non-zero): the other
+// query tile's softmax warps may then start theirs, so that the two tiles use the
+// special-function unit out of phase and one tile's loads / maxima / stores overlap the other
+// tile's exponentials.
 template <bool MASK>
 __device__ __forceinline__ float store_probabilities(uint32_t tS, int valid, float c, float m,
-                                                     const uint32_t (&s)[kBH]) {
+                                                     const uint32_t (&s)[kBH], uint32_t turn_bar,
+                                                     int lane) {
     float sum[4] = {0.f, 0.f, 0.f, 0.f};
     uint32_t pk[kBH / 2];
 #pragma unroll
@@ -131,6 +137,7 @@ __device__ __forceinline__ float store_probabilities(uint32_t tS, int valid, flo
         if (MASK && 2 * i + 1 >= valid) p1 = 0.f;
         sum[i & 3] += p0 + p1;
         pk[i] = pack_bf16x2(p0, p1);
+        if (i == kBH / 4 - 1 && turn_bar != 0 && lane == 0) ptx::mbar_arrive(turn_bar);
     }
     ptx::tmem_st32(tS, pk);
     return (sum[0] + sum[1]) + (sum[2] + sum[3]);
@@ -189,6 +196,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
             }
             ptx::mbar_init(ptx::smem_addr(&ctrl->o_done[t]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctrl->o_final[t]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->turn[t]), kBM / 32);
         }
         ctrl->abort_flag = 0;
         ptx::fence_barrier_init();
@@ -397,8 +405,19 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                     l *= alpha;
                     m = m_new;
                 }
-                l += (vh == kBH) ? store_probabilities<false>(tS, vh, c, m, s)
-                                 : store_probabilities<true>(tS, vh, c, m, s);
+                uint32_t turn_bar = 0;
+                if (ntq == 2) {
+                    // tile 0 starts half ph once tile 1 is half way through half ph - 1; tile 1
+                    // starts half ph once tile 0 is half way through half ph
+                    turn_bar = ptx::smem_addr(&ctrl->turn[t ^ 1]);
+                    if (t == 1 || ph > 0) {
+                        ok = wait_bar(ptx::smem_addr(&ctrl->turn[t]), (ph - 1 + t) & 1, abort_flag,
+                                      p.dev_status);
+                        if (!ok) break;
+                    }
+                }
+                l += (vh == kBH) ? store_probabilities<false>(tS, vh, c, m, s, turn_bar, lane)
+                                 : store_probabilities<true>(tS, vh, c, m, s, turn_bar, lane);
                 ptx::tmem_wait_st();
                 if (hh == 0 && valid < kBN) {
                     // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
