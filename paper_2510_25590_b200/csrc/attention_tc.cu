@@ -11,22 +11,24 @@
 //              are two tensor maps walked one after the other
 //   warps 9,10 tcgen05.mma issuers, one per query tile (the whole warp walks the
 //              loop, one elected lane issues); warp 9 owns the tensor-memory allocation
+//   warp  11   idle (fills the third warpgroup so that registers can be moved from
+//              it to the softmax warpgroups with setmaxnreg)
 //
-// Tensor memory (512 columns): S0a S0b | S1a S1b | O0 | O1.  The logits of a
-// query tile are produced 64 keys at a time, S_t(h) = Q_t K_h^T (fp32, 64
-// columns), alternating between the tile's two buffers a / b.  The softmax
-// warps read S_t(h) back, write the probabilities over it as packed bf16 (P
-// aliases the first 32 columns of its S buffer) and O_t += P_t(h) V_h runs
-// straight from tensor memory.  Because S_t(h+1) sits in the other buffer and
-// is issued before P_t(h) exists, a softmax warp never waits for its own
-// P*V product: the chain S -> softmax -> P*V -> next S of the one-buffer
-// scheme is cut, and the special-function unit (exp2) stays busy.
+// Tensor memory (512 columns): S0 | S1 | O0 | O1.  S_t = Q_t K_j^T (fp32, 128
+// columns) is read back by the softmax warps of tile t, the probabilities are
+// written over it as packed bf16 (P aliases the first 64 columns of S) in two
+// chunks of 64 keys, and O_t += P_t V_j runs straight from tensor memory: the
+// product of the first chunk is issued while the exponentials of the second
+// are still being computed.  Each query tile has its own issuer warp, so the
+// dependency chain of a tile (S -> softmax -> P*V -> next S) only stalls that
+// tile; the other tile's products fill the tensor pipe meanwhile.  The two
+// tiles take turns on the special-function unit (exp2), which keeps them out
+// of phase.
 //
 // Online softmax in the exp2 domain; O is rescaled in tensor memory only when
-// a row maximum grows by more than 2^8 (after waiting for the P*V products
-// already issued for that tile).  Keys past a segment's live count are masked
-// in the softmax and their V rows zeroed in shared memory, so garbage (even
-// NaN) behind the live prefix cannot leak.
+// a row maximum grows by more than 2^8.  Keys past a segment's live count are
+// masked in the softmax and their V rows zeroed in shared memory, so garbage
+// (even NaN) behind the live prefix cannot leak.
 //
 // Occupancy: the key tiles of one (request, head, query pair) can be split over
 // several CTAs (split-KV).  Each split then writes its unnormalised output and
@@ -44,10 +46,10 @@
 
 namespace regione {
 
-constexpr int kAttnThreads = 352;
+constexpr int kAttnThreads = 384;        // 2 softmax warpgroups + 1 of producer / issuers
 constexpr int kBM = 128;                 // query rows per tile
 constexpr int kBN = 128;                 // key rows per shared-memory tile
-constexpr int kBH = 64;                  // key rows per S buffer (half a tile)
+constexpr int kBH = 64;                  // key rows per P chunk (half a tile)
 constexpr int kHalfBytes = 128 * 64 * 2; // one 128-row x 64-column bf16 box (128-byte rows)
 constexpr long long kTimeoutCycles = 4000000000LL;
 
@@ -64,11 +66,10 @@ struct AttnCtrl {
     uint64_t q_full;
     uint64_t kv_full[6];
     uint64_t kv_empty[6];
-    uint64_t s_full[2][2];      // [query tile][S buffer]
-    uint64_t p_full[2][2];
-    uint64_t o_done[2];         // one completion per P*V product of the tile
+    uint64_t s_full[2];         // [query tile]
+    uint64_t p_full[2][2];      // [query tile][chunk of 64 keys]
     uint64_t o_final[2];        // completes once, after the tile's last P*V product
-    uint64_t turn[2];           // turn[t]: the other tile is half way through its exponentials
+    uint64_t turn[2];           // turn[t]: the other query tile has finished a tile's exponentials
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -102,12 +103,9 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
-// Row maximum (times the scale, exp2 domain) of the 64 logits of one S buffer; `s` keeps them.
+// Maximum of 64 logits held in registers (keys >= valid masked out).
 template <bool MASK>
-__device__ __forceinline__ float load_logits_max(uint32_t tS, int valid, float c, uint32_t (&s)[kBH]) {
-    ptx::tmem_ld32(tS, s);
-    ptx::tmem_ld32(tS + 32, s + 32);
-    ptx::tmem_wait_ld();
+__device__ __forceinline__ float chunk_max(const uint32_t* s, int valid) {
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
     for (int i = 0; i < kBH; ++i) {
@@ -115,18 +113,14 @@ __device__ __forceinline__ float load_logits_max(uint32_t tS, int valid, float c
         if (MASK && i >= valid) v = -INFINITY;
         mx[i & 3] = fmaxf(mx[i & 3], v);
     }
-    return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
+    return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 }
 
-// p = 2^(s*c - m) for the 64 logits, written over S as packed bf16; returns their fp32 sum.
-// After the first half of the exponentials lane 0 arrives on `turn_bar` (if non-zero): the other
-// query tile's softmax warps may then start theirs, so that the two tiles use the
-// special-function unit out of phase and one tile's loads / maxima / stores overlap the other
-// tile's exponentials.
+// p = 2^(s*c - m) for 64 logits, written to tensor memory at `tP` (32 columns) as packed bf16;
+// returns their fp32 sum.
 template <bool MASK>
-__device__ __forceinline__ float store_probabilities(uint32_t tS, int valid, float c, float m,
-                                                     const uint32_t (&s)[kBH], uint32_t turn_bar,
-                                                     int lane) {
+__device__ __forceinline__ float chunk_probabilities(uint32_t tP, const uint32_t* s, int valid,
+                                                     float c, float m) {
     float sum[4] = {0.f, 0.f, 0.f, 0.f};
     uint32_t pk[kBH / 2];
 #pragma unroll
@@ -137,9 +131,8 @@ __device__ __forceinline__ float store_probabilities(uint32_t tS, int valid, flo
         if (MASK && 2 * i + 1 >= valid) p1 = 0.f;
         sum[i & 3] += p0 + p1;
         pk[i] = pack_bf16x2(p0, p1);
-        if (i == kBH / 4 - 1 && turn_bar != 0 && lane == 0) ptx::mbar_arrive(turn_bar);
     }
-    ptx::tmem_st32(tS, pk);
+    ptx::tmem_st32(tP, pk);
     return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
@@ -190,11 +183,9 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
             ptx::mbar_init(ptx::smem_addr(&ctrl->kv_empty[s]), ntq);    // one commit per issuer
         }
         for (int t = 0; t < 2; ++t) {
-            for (int u = 0; u < 2; ++u) {
-                ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t][u]), 1);
-                ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t][u]), kBM / 32);
-            }
-            ptx::mbar_init(ptx::smem_addr(&ctrl->o_done[t]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t][0]), kBM / 32);
+            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t][1]), kBM / 32);
             ptx::mbar_init(ptx::smem_addr(&ctrl->o_final[t]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctrl->turn[t]), kBM / 32);
         }
@@ -210,7 +201,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     ptx::tc_fence_after_sync();
     const uint32_t tmem = ctrl->tmem_base;
 
-    // key tile jl of this CTA -> (segment, first row, live rows); a tile yields one S half when
+    // key tile jl of this CTA -> (segment, first row, live rows); a tile yields one P chunk when
     // at most 64 of its keys are live, else two
     auto tile_seg = [&](int jl, bool& cached, int& row0, int& valid) {
         const int j = j_first + jl;
@@ -219,12 +210,13 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         row0 = jj * kBN;
         valid = min(kBN, (cached ? nc : nf) - row0);
     };
-    auto tile_halves = [&](int jl) {
+    auto tile_chunks = [&](int jl) {
         bool cached; int row0, valid;
         tile_seg(jl, cached, row0, valid);
         return valid > kBH ? 2 : 1;
     };
 
+    if (warp >= 8) ptx::reg_dealloc<56>();              // producer / issuer warpgroup gives registers up
     if (warp == 8) {
         // ================= TMA producer =================
         if (lane == 0) {
@@ -257,12 +249,10 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
     } else if (warp == 9 || warp == 10) {
         // ================= MMA issuers: warp 9 for query tile 0, warp 10 for query tile 1 ========
-        // Each whole warp walks its loop and waits on the barriers; one elected lane issues.  Two
-        // independent issuers keep the tensor pipe fed: while one sits in the fixed latency of a
-        // barrier wait or a commit, the products of the other execute.
+        // Each whole warp walks its loop and waits on the barriers; one elected lane issues.
         const int t = warp - 9;
         if (t < ntq) {
-            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBH, false);
+            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
             constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
             // K-major operands (Q, K): 128-byte swizzle, LBO unused; V is MN-major: 64-column
@@ -270,183 +260,183 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
             const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
             const uint32_t k_lo = ptx::smem_desc_lo(sKV, 16);
             const uint32_t v_lo = ptx::smem_desc_lo(sKV, kHalfBytes);
-            const uint32_t tS0 = tmem + t * kBN, tOt = tmem + 256 + t * D;
-            // S_t(buffer u) = Q_t K[64 hh .. 64 hh + 64)^T
-            auto issue_s = [&](int stage, int hh, int u) {
-                const uint32_t b0 = k_lo + ((stage * kTileBytes + hh * (kBH * 128)) >> 4);
+            const uint32_t tSt = tmem + t * kBN, tOt = tmem + 256 + t * D;
+            // S_t = Q_t K^T
+            auto issue_s = [&](int stage) {
+                const uint32_t b0 = k_lo + ((stage * kTileBytes) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
-                    ptx::mma_ss(tS0 + u * kBH, ptx::smem_desc_join(q_lo + off, hi_k),
+                    ptx::mma_ss(tSt, ptx::smem_desc_join(q_lo + off, hi_k),
                                 ptx::smem_desc_join(b0 + off, hi_k), idesc_s, kk > 0);
                 }
             };
-            // O_t (+)= P_t(buffer u) V[64 hh .. 64 hh + 64) : A from tensor memory (bf16 pairs,
+            // O_t (+)= P_t[chunk] V[64 chunk .. 64 chunk + 64) : A from tensor memory (bf16 pairs,
             // 8 columns per 16 keys)
-            auto issue_pv = [&](int stage, int hh, int u, bool accumulate) {
-                const uint32_t b0 = v_lo + ((stage * kTileBytes + hh * (kBH / 16) * 2048) >> 4);
+            auto issue_pv = [&](int stage, int chunk, bool accumulate) {
+                const uint32_t b0 = v_lo + ((stage * kTileBytes + chunk * (kBH / 16) * 2048) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < kBH / 16; ++kk)
-                    ptx::mma_ts(tOt, tS0 + u * kBH + kk * 8,
+                    ptx::mma_ts(tOt, tSt + chunk * (kBH / 2) + kk * 8,
                                 ptx::smem_desc_join(b0 + ((kk * 2048) >> 4), hi_k), idesc_pv,
                                 (accumulate || kk > 0) ? 1u : 0u);
             };
-            // cursor of the next S half to issue: key tile sj, half shh
-            int sj = 0, shh = 0;
-            int s_halves = n_tiles > 0 ? tile_halves(0) : 0;
-            auto s_stage = [&]() { return (2 * sj) % kStages; };
-            auto s_parity = [&]() { return ((2 * sj) / kStages) & 1; };
-            auto s_advance = [&]() {
-                if (++shh == s_halves) {
-                    shh = 0;
-                    ++sj;
-                    s_halves = sj < n_tiles ? tile_halves(sj) : 0;
-                }
-            };
             bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
-            // prologue: the first two S halves
-            for (int pre = 0; pre < 2 && ok && sj < n_tiles; ++pre) {
-                if (shh == 0)
-                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[s_stage()]), s_parity(), abort_flag,
+            if (ok && n_tiles > 0) {
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[0]), 0, abort_flag, p.dev_status);
+                if (ok) {
+                    ptx::tc_fence_after_sync();
+                    if (ptx::elect_one()) {
+                        issue_s(0);
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[0]));
+                    }
+                    __syncwarp();
+                }
+            }
+            int nb = 0;                                     // second chunks seen so far
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int iv = 2 * j + 1, ik = 2 * j + 2;
+                const int sv = iv % kStages, sk = ik % kStages;
+                const bool more = (j + 1 < n_tiles);
+                const int chunks = tile_chunks(j);
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                              p.dev_status);
+                if (ok)
+                    ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][0]), j & 1, abort_flag,
                                   p.dev_status);
+                if (!ok) break;
+                if (chunks == 2) {
+                    ptx::tc_fence_after_sync();
+                    if (ptx::elect_one()) issue_pv(sv, 0, j > 0);
+                    __syncwarp();
+                }
+                if (more)
+                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / kStages) & 1, abort_flag,
+                                  p.dev_status);
+                if (ok && chunks == 2) {
+                    ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][1]), nb & 1, abort_flag,
+                                  p.dev_status);
+                    ++nb;
+                }
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 if (ptx::elect_one()) {
-                    issue_s(s_stage(), shh, pre);
-                    ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t][pre]));
-                    if (shh == s_halves - 1)
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[s_stage()]));
+                    issue_pv(sv, chunks - 1, j > 0 || chunks == 2);
+                    if (!more) ptx::mma_commit(ptx::smem_addr(&ctrl->o_final[t]));
+                    ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sv]));
+                    if (more) {
+                        issue_s(sk);
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk]));
+                    }
                 }
                 __syncwarp();
-                s_advance();
-            }
-            int ph = 0;                                     // running index of the P*V half
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int iv = 2 * j + 1, sv = iv % kStages;
-                const int halves = tile_halves(j);
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
-                              p.dev_status);
-                for (int hh = 0; hh < halves && ok; ++hh, ++ph) {
-                    const int u = ph & 1;
-                    const bool more = sj < n_tiles;         // S half ph + 2 exists
-                    if (more && shh == 0)
-                        ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[s_stage()]), s_parity(),
-                                      abort_flag, p.dev_status);
-                    if (ok)
-                        ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][u]), (ph >> 1) & 1, abort_flag,
-                                      p.dev_status);
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    if (ptx::elect_one()) {
-                        issue_pv(sv, hh, u, ph > 0);
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->o_done[t]));
-                        if (j == n_tiles - 1 && hh == halves - 1)
-                            ptx::mma_commit(ptx::smem_addr(&ctrl->o_final[t]));
-                        if (hh == halves - 1) ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sv]));
-                        if (more) {
-                            issue_s(s_stage(), shh, u);
-                            ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t][u]));
-                            if (shh == s_halves - 1)
-                                ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[s_stage()]));
-                        }
-                    }
-                    __syncwarp();
-                    if (more) s_advance();
-                }
             }
         }
     } else if (warp < 4 * ntq) {
         // ================= softmax / correction / epilogue =================
+        ptx::reg_alloc<224>();                              // a row of 128 logits stays in registers
         const int t = warp >> 2;
         const int row = ((warp & 3) << 5) + lane;                  // row of the query tile
         const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
-        const uint32_t tSt = tmem + lane_sel + t * kBN;
+        const uint32_t tS = tmem + lane_sel + t * kBN;
         const uint32_t tO = tmem + lane_sel + 256 + t * D;
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
-        int ph = 0;                                                // running half index
-        for (int j = 0; j < n_tiles && ok; ++j) {
+        for (int j = 0; j < n_tiles; ++j) {
             bool cached; int row0, valid;
             tile_seg(j, cached, row0, valid);
-            const int halves = valid > kBH ? 2 : 1;
-            for (int hh = 0; hh < halves; ++hh, ++ph) {
-                const int u = ph & 1;
-                const uint32_t tS = tSt + u * kBH;
-                ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t][u]), (ph >> 1) & 1, abort_flag,
+            const int chunks = valid > kBH ? 2 : 1;
+            ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            // (P_t V_{j-1} has completed here: S_t(j) was issued after it by the same thread and
+            // tcgen05.mma executes in issue order, so O_t may be rescaled and P_t overwritten)
+            uint32_t s[kBN];
+            ptx::tmem_ld32(tS, s);
+            ptx::tmem_ld32(tS + 32, s + 32);
+            ptx::tmem_wait_ld();
+            float mt;
+            if (chunks == 2) {
+                ptx::tmem_ld32(tS + 64, s + 64);
+                ptx::tmem_ld32(tS + 96, s + 96);
+                mt = chunk_max<false>(s, kBH);
+                ptx::tmem_wait_ld();
+                mt = fmaxf(mt, valid == kBN ? chunk_max<false>(s + kBH, kBH)
+                                            : chunk_max<true>(s + kBH, valid - kBH));
+            } else {
+                mt = valid == kBH ? chunk_max<false>(s, kBH) : chunk_max<true>(s, valid);
+            }
+            mt *= c;
+            if (j == 0) {
+                m = mt;
+            } else if (__any_sync(0xffffffffu, mt > m + 8.f)) {
+                const float m_new = fmaxf(m, mt);
+                const float alpha = fast_exp2(m - m_new);
+                uint32_t r[32];
+#pragma unroll 1
+                for (int ch = 0; ch < D / 32; ++ch) {
+                    ptx::tmem_ld32(tO + ch * 32, r);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                    ptx::tmem_st32(tO + ch * 32, r);
+                }
+                l *= alpha;
+                m = m_new;
+            }
+            // The two query tiles take turns on the special-function unit: tile 1 computes the
+            // exponentials of key tile j after tile 0 has finished its own, tile 0 those of key
+            // tile j + 1 after tile 1 has finished j.  Run alone they take half as long, which
+            // shortens each tile's chain S -> softmax -> P*V -> next S; the other tile's loads,
+            // maxima and products fall into the gap.
+            if (ntq == 2 && (t == 1 || j > 0)) {
+                ok = wait_bar(ptx::smem_addr(&ctrl->turn[t]), (j - 1 + t) & 1, abort_flag,
                               p.dev_status);
                 if (!ok) break;
-                ptx::tc_fence_after_sync();
-                const int vh = min(kBH, valid - hh * kBH);         // live keys of this half (>= 1)
-                uint32_t s[kBH];
-                const float mt = (vh == kBH) ? load_logits_max<false>(tS, vh, c, s)
-                                             : load_logits_max<true>(tS, vh, c, s);
-                if (ph == 0) {
-                    m = mt;
-                } else if (__any_sync(0xffffffffu, mt > m + 8.f)) {
-                    // raise the reference maximum: every P*V product issued so far for this tile
-                    // (halves 0 .. ph-1) must have landed in O before O is rescaled
-                    ok = wait_bar(ptx::smem_addr(&ctrl->o_done[t]), (ph - 1) & 1, abort_flag,
-                                  p.dev_status);
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    const float m_new = fmaxf(m, mt);
-                    const float alpha = fast_exp2(m - m_new);
-                    uint32_t r[32];
+            }
+            // first chunk of probabilities (keys 0..63 of the tile)
+            l += (valid >= kBH) ? chunk_probabilities<false>(tS, s, kBH, c, m)
+                                : chunk_probabilities<true>(tS, s, valid, c, m);
+            if (chunks == 1 && ntq == 2 && lane == 0)
+                ptx::mbar_arrive(ptx::smem_addr(&ctrl->turn[t ^ 1]));
+            ptx::tmem_wait_st();
+            if (valid < kBN) {
+                // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
+                const int iv = 2 * j + 1, sv = iv % kStages;
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                              p.dev_status);
+                if (!ok) break;
+                if (row >= valid) {
+                    uint8_t* vrow = smem_gen + 2 * kTileBytes + sv * kTileBytes + row * 128;
 #pragma unroll
-                    for (int ch = 0; ch < D / 32; ++ch) {
-                        ptx::tmem_ld32(tO + ch * 32, r);
-                        ptx::tmem_wait_ld();
+                    for (int hf = 0; hf < Cfg::kHalves; ++hf)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        ptx::tmem_st32(tO + ch * 32, r);
-                    }
-                    l *= alpha;
-                    m = m_new;
+                        for (int q = 0; q < 8; ++q)
+                            reinterpret_cast<uint4*>(vrow + hf * kHalfBytes)[q] = make_uint4(0, 0, 0, 0);
                 }
-                uint32_t turn_bar = 0;
-                if (ntq == 2) {
-                    // tile 0 starts half ph once tile 1 is half way through half ph - 1; tile 1
-                    // starts half ph once tile 0 is half way through half ph
-                    turn_bar = ptx::smem_addr(&ctrl->turn[t ^ 1]);
-                    if (t == 1 || ph > 0) {
-                        ok = wait_bar(ptx::smem_addr(&ctrl->turn[t]), (ph - 1 + t) & 1, abort_flag,
-                                      p.dev_status);
-                        if (!ok) break;
-                    }
-                }
-                l += (vh == kBH) ? store_probabilities<false>(tS, vh, c, m, s, turn_bar, lane)
-                                 : store_probabilities<true>(tS, vh, c, m, s, turn_bar, lane);
+                ptx::fence_proxy_async_smem();
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t][0]));
+            if (chunks == 2) {
+                // second chunk (keys 64..127) while the first chunk's product runs
+                l += (valid == kBN) ? chunk_probabilities<false>(tS + kBH / 2, s + kBH, kBH, c, m)
+                                    : chunk_probabilities<true>(tS + kBH / 2, s + kBH, valid - kBH, c, m);
+                if (ntq == 2 && lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->turn[t ^ 1]));
                 ptx::tmem_wait_st();
-                if (hh == 0 && valid < kBN) {
-                    // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
-                    const int iv = 2 * j + 1, sv = iv % kStages;
-                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
-                                  p.dev_status);
-                    if (!ok) break;
-                    if (row >= valid) {
-                        uint8_t* vrow = smem_gen + 2 * kTileBytes + sv * kTileBytes + row * 128;
-#pragma unroll
-                        for (int hf = 0; hf < Cfg::kHalves; ++hf)
-#pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                reinterpret_cast<uint4*>(vrow + hf * kHalfBytes)[q] = make_uint4(0, 0, 0, 0);
-                    }
-                    ptx::fence_proxy_async_smem();
-                }
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t][u]));
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t][1]));
             }
         }
-        const int n_halves = ph;
         // epilogue (rows past n_q are not written)
         const int qrow = q0 + t * kBM + row;
         const bool live = qrow < nq;
-        if (n_halves > 0 && ok) {
-            // (o_done advances one phase per product and can be one or two phases short of the
-            // end here, which a parity wait cannot tell apart: hence the barrier of its own)
+        if (n_tiles > 0 && ok) {
             ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status);
             if (ok) ptx::tc_fence_after_sync();
         }

@@ -24,6 +24,15 @@ __device__ __forceinline__ uint32_t elect_one() {
     return pred;
 }
 
+// Register re-balancing between warp-specialised roles: every warp of a warpgroup (4 aligned
+// warps) executes the same instruction; `inc` waits until other warpgroups have released enough.
+template <int N> __device__ __forceinline__ void reg_alloc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void reg_dealloc() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 // ---- mbarrier -----------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
