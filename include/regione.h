@@ -185,6 +185,37 @@ int regione_region_attention(const regione_bf16* q,
                              int32_t* dev_status, void* stream);
 
 /*
+ * Region attention that brings its own scratch memory.  (The paper has no
+ * counterpart: this entry point exists only for the way the library is deployed.)
+ *
+ * Same computation, arguments and limits as regione_region_attention, without the
+ * workspace pair.  It is meant for callers that cannot obtain device memory at the
+ * point of the call: an inference server that hands all of HBM to its own arena at
+ * start-up so a later cudaMalloc fails, or a denoising loop that must not stall,
+ * since cudaMalloc / cudaFree synchronise the whole device.  The split-KV partials
+ * go to a 64 MiB array compiled into the library (device memory that every GPU
+ * loading the library holds until the process ends); the call performs no
+ * allocation of any kind.
+ *
+ *  - A shape whose partials would not fit, i.e.
+ *    regione_region_attention_workspace(...) > 64 MiB, is refused with
+ *    REGIONE_WORKSPACE_TOO_SMALL; nothing is launched.
+ *  - The first call on each device looks the array's device address up (with that
+ *    device current) and remembers it.  Make that first call outside any stream
+ *    capture.
+ *  - All calls on a device share the one array and it keeps whatever the last call
+ *    left in it.  Nothing in it needs clearing between calls, but two calls whose
+ *    kernels overlap on the GPU (different streams) race on it: serialise them.
+ */
+int regione_region_attention_static(const regione_bf16* q,
+                                    const regione_bf16* k_fresh, const regione_bf16* v_fresh,
+                                    const regione_bf16* k_cache, const regione_bf16* v_cache,
+                                    const int32_t* n_q, const int32_t* n_fresh, const int32_t* n_cache,
+                                    int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D,
+                                    float softmax_scale, regione_bf16* out,
+                                    int32_t* dev_status, void* stream);
+
+/*
  * One step of the AVDCache criterion (Sec. 4, "Adaptive Velocity Decay Cache",
  * the decay-factor and criterion equations).  Pure host arithmetic:
  *     p = *running_product * (1 - dt) * gamma

@@ -34,6 +34,7 @@ SIGNATURES = {
     "regione_rikv_store": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
     "regione_region_attention_workspace": (c_size_t, [c_int] * 6),
     "regione_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, c_size_t, _P, _P]),
+    "regione_region_attention_static": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, _P]),
     "regione_avd_step": (c_int, [POINTER(c_double), c_double, c_double, c_double, POINTER(c_int)]),
     "regione_velocity_decay": (c_int, [_P, c_float, c_float, _P, _P, _P, c_int, c_int, c_int, _P, _P]),
     "regione_merge": (c_int, [_P, _P, _P, _P, c_float, c_int, c_int, c_int, c_int, _P, _P, _P]),
@@ -197,6 +198,27 @@ def region_attention(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cach
         _ptr(n_cache, i32), B, Nq_cap, Nf_cap, Nc_cap, H, D, float(softmax_scale), _ptr(out, bf, "out"),
         _ptr(workspace, None, "workspace"), ws_bytes, _ptr(dev_status, i32), _stream(stream)),
         "regione_region_attention")
+
+
+def region_attention_static(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, out,
+                            softmax_scale=0.0, dev_status=None, stream=None):
+    """Region attention with the library's built-in 64 MiB scratch: no workspace, no allocation.
+
+    For callers that cannot allocate device memory where they call (all of HBM already owned by
+    an arena, or a loop that must not hit the device-wide synchronisation of cudaMalloc).  Calls
+    on one device share the scratch, so do not let two of them overlap on the GPU.
+    """
+    torch = _torch()
+    bf = torch.bfloat16
+    B, Nq_cap, H, D = q.shape
+    Nf_cap = 0 if k_fresh is None else k_fresh.shape[1]
+    Nc_cap = 0 if k_cache is None else k_cache.shape[1]
+    i32 = torch.int32
+    _check(load().regione_region_attention_static(
+        _ptr(q, bf, "q"), _ptr(k_fresh, bf, "k_fresh"), _ptr(v_fresh, bf, "v_fresh"),
+        _ptr(k_cache, bf, "k_cache"), _ptr(v_cache, bf, "v_cache"), _ptr(n_q, i32), _ptr(n_fresh, i32),
+        _ptr(n_cache, i32), B, Nq_cap, Nf_cap, Nc_cap, H, D, float(softmax_scale), _ptr(out, bf, "out"),
+        _ptr(dev_status, i32), _stream(stream)), "regione_region_attention_static")
 
 
 def avd_step(running_product: float, dt: float, gamma: float, delta: float):

@@ -681,4 +681,63 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
     return D == 64 ? launch_tc<64>(maps, prm, B, st) : launch_tc<128>(maps, prm, B, st);
 }
 
+// ---- variant with library-owned scratch -----------------------------------------------------
+// The split-KV partials of regione_region_attention_static live here instead of in a caller
+// workspace.  The array is part of the library image: every GPU that loads the library keeps
+// these bytes resident until the process exits.
+constexpr size_t kStaticScratchBytes = (size_t)64 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};      // device address of the array, per device
+}  // namespace
+
+// Device address of g_static_scratch on the current device (in host code the symbol itself is
+// only a stand-in and must never be handed to a kernel).  Resolved on the first call per device.
+static int static_scratch_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return REGIONE_CUDA_ERROR;
+    void* addr = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (addr == nullptr) {
+        if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || addr == nullptr) {
+            (void)cudaGetLastError();
+            return REGIONE_CUDA_ERROR;
+        }
+        __atomic_store_n(&g_static_scratch_addr[dev], addr, __ATOMIC_RELEASE);
+    }
+    *out = addr;
+    return REGIONE_OK;
+}
+
 }  // namespace regione
+
+extern "C" int regione_region_attention_static(
+    const regione_bf16* q, const regione_bf16* k_fresh, const regione_bf16* v_fresh,
+    const regione_bf16* k_cache, const regione_bf16* v_cache, const int32_t* n_q,
+    const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap, int Nf_cap, int Nc_cap, int H,
+    int D, float softmax_scale, regione_bf16* out, int32_t* dev_status, void* stream) {
+    using namespace regione;
+    if (!q || !out || !n_q || !n_fresh || !n_cache) return REGIONE_INVALID_ARG;
+    if (B < 0 || Nq_cap < 0 || Nf_cap < 0 || Nc_cap < 0 || H < 1) return REGIONE_INVALID_ARG;
+    if (Nf_cap > 0 && (!k_fresh || !v_fresh)) return REGIONE_INVALID_ARG;
+    if (Nc_cap > 0 && (!k_cache || !v_cache)) return REGIONE_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_fresh) || !aligned16(v_fresh) ||
+        !aligned16(k_cache) || !aligned16(v_cache))
+        return REGIONE_INVALID_ARG;
+    if (D != 64 && D != 128) return REGIONE_UNSUPPORTED;
+    if (B > 65535 || H > 65535) return REGIONE_UNSUPPORTED;
+    if (B == 0 || Nq_cap == 0) return REGIONE_OK;
+    // the partials of this shape must fit the fixed array: refuse, never truncate
+    const size_t need = region_attention_tc_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D);
+    if (need > kStaticScratchBytes) return REGIONE_WORKSPACE_TOO_SMALL;
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != REGIONE_OK) return rc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    // Nothing in the scratch has to start at zero: every word the merge kernel reads is written
+    // by the attention kernel of the same call, so the previous call's contents are harmless.
+    return launch_region_attention_tc(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
+                                      B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, scratch,
+                                      kStaticScratchBytes, dev_status, (cudaStream_t)stream);
+}
