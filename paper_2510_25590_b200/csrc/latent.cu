@@ -41,29 +41,52 @@ velocity_decay_kernel(const uint4* __restrict__ v_in, float neg_dt_scale, uint4*
     if (v_cache_out != nullptr) v_cache_out[off] = v;
 }
 
-// x_out[n] = slot[n] >= 0 ? x_e[slot[n]] : x_full[n] - dt * v_last[n].  One thread = 8 channels.
+// x_out[n] = slot[n] >= 0 ? x_e[slot[n]] : x_full[n] - dt * v_last[n].  One thread = kMergeUnroll
+// chunks of 8 channels, blockDim apart; all slots are read first, then every data load is issued
+// before the first store, so several independent loads per thread are in flight.
+constexpr int kMergeUnroll = 4;
+
 __global__ void __launch_bounds__(kLatThreads)
 merge_kernel(const uint4* x_full, const uint4* __restrict__ v_last,
              const uint4* __restrict__ x_e, const int32_t* __restrict__ slot, float neg_dt, int N,
              int Ne_cap, int cpr, uint4* x_out, int32_t* dev_status) {
     const int b = blockIdx.y;
     const unsigned total = (unsigned)N * (unsigned)cpr;
-    const unsigned e = blockIdx.x * (unsigned)kLatThreads + threadIdx.x;
-    if (e >= total) return;
-    const unsigned n = e / (unsigned)cpr;
-    const unsigned c = e - n * (unsigned)cpr;
-    const int s = slot[(size_t)b * N + n];
-    const size_t off = (size_t)b * N * cpr + e;
-    if (s >= 0) {
-        if (s >= Ne_cap) {
-            record_status(dev_status, REGIONE_DEV_BOUNDS);
-            return;
+    const unsigned base = blockIdx.x * (unsigned)(kLatThreads * kMergeUnroll) + threadIdx.x;
+    const size_t req = (size_t)b * N * cpr;
+    int s[kMergeUnroll];
+    unsigned c[kMergeUnroll];
+#pragma unroll
+    for (int u = 0; u < kMergeUnroll; ++u) {
+        const unsigned e = base + (unsigned)u * kLatThreads;
+        s[u] = -2;                                   // -2: past the end, nothing to do
+        if (e < total) {
+            const unsigned n = e / (unsigned)cpr;
+            c[u] = e - n * (unsigned)cpr;
+            const int sv = slot[(size_t)b * N + n];
+            s[u] = sv < 0 ? -1 : sv;                 // any negative slot means "unedited"
+            if (s[u] >= Ne_cap) {
+                record_status(dev_status, REGIONE_DEV_BOUNDS);
+                s[u] = -2;
+            }
         }
-        x_out[off] = ldg128(x_e + ((size_t)b * Ne_cap + s) * cpr + c);
-    } else {
-        const uint4 x = x_full[off];
-        const uint4 v = ld_stream128(v_last + off);
-        x_out[off] = axpy8(x, v, neg_dt);
+    }
+    uint4 x[kMergeUnroll], v[kMergeUnroll];
+#pragma unroll
+    for (int u = 0; u < kMergeUnroll; ++u) {
+        const size_t off = req + base + (size_t)u * kLatThreads;
+        if (s[u] >= 0) {
+            x[u] = ldg128(x_e + ((size_t)b * Ne_cap + s[u]) * cpr + c[u]);
+        } else if (s[u] == -1) {
+            x[u] = x_full[off];
+            v[u] = ld_stream128(v_last + off);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kMergeUnroll; ++u) {
+        const size_t off = req + base + (size_t)u * kLatThreads;
+        if (s[u] >= 0) x_out[off] = x[u];
+        else if (s[u] == -1) x_out[off] = axpy8(x[u], v[u], neg_dt);
     }
 }
 
@@ -103,7 +126,8 @@ extern "C" int regione_merge(const regione_bf16* x_full, const regione_bf16* v_l
     const long long cpr = C / 8, total = (long long)N * cpr;
     if (total + kLatThreads >= 0x7fffffffLL) return REGIONE_UNSUPPORTED;
     if (B == 0) return REGIONE_OK;
-    dim3 grid((unsigned)((total + kLatThreads - 1) / kLatThreads), B);
+    const long long per_block = (long long)kLatThreads * kMergeUnroll;
+    dim3 grid((unsigned)((total + per_block - 1) / per_block), B);
     merge_kernel<<<grid, kLatThreads, 0, (cudaStream_t)stream>>>(
         (const uint4*)x_full, (const uint4*)v_last_full, (const uint4*)x_e, slot, -dt_unedited, N,
         Ne_cap, (int)cpr, (uint4*)x_out, dev_status);

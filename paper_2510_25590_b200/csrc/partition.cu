@@ -20,8 +20,7 @@ namespace cg = cooperative_groups;
 
 namespace regione {
 
-constexpr int kPartThreads = 256;
-constexpr int kPartWarps = kPartThreads / 32;
+constexpr int kPartMaxThreads = 512;         // block size grows with the tokens per CTA
 constexpr int kPartMaxWords = 4096;          // 131072 tokens per CTA
 constexpr int kPartMaxCluster = 8;
 
@@ -84,8 +83,31 @@ __device__ void emit_indices(const uint32_t* bits, const int* prefix, int start,
     }
 }
 
+// Adds one 16-byte chunk (8 channels) of a token to its partial sums: x0_hat = x_t - t v, then
+// cosine terms (dot, |x0_hat|^2, |ref|^2) or the squared distance.
+__device__ __forceinline__ void accumulate_chunk(uint4 xv, uint4 vv, uint4 rv, float t, int metric,
+                                                 float& a0, float& a1, float& a2) {
+    const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
+    const uint32_t vs[4] = {vv.x, vv.y, vv.z, vv.w};
+    const uint32_t rs[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float h0 = fmaf(-t, bf16_lo(vs[k]), bf16_lo(xs[k]));
+        const float h1 = fmaf(-t, bf16_hi(vs[k]), bf16_hi(xs[k]));
+        const float r0 = bf16_lo(rs[k]), r1 = bf16_hi(rs[k]);
+        if (metric == REGIONE_METRIC_COSINE) {
+            a0 = fmaf(h0, r0, a0); a0 = fmaf(h1, r1, a0);
+            a1 = fmaf(h0, h0, a1); a1 = fmaf(h1, h1, a1);
+            a2 = fmaf(r0, r0, a2); a2 = fmaf(r1, r1, a2);
+        } else {
+            const float d0 = h0 - r0, d1 = h1 - r1;
+            a0 = fmaf(d0, d0, a0); a0 = fmaf(d1, d1, a0);
+        }
+    }
+}
+
 template <int L>
-__global__ void __launch_bounds__(kPartThreads)
+__global__ void __launch_bounds__(kPartMaxThreads)
 partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ v,
                  const uint16_t* __restrict__ ref, int N, int C, int share, float t, int metric,
                  float threshold, uint8_t* __restrict__ mask, int32_t* __restrict__ edit_idx,
@@ -110,57 +132,60 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
     const size_t req = (size_t)b * N;
 
     // ---- phase 1: score + decision, one mask word per 32 tokens -------------------------
-    for (int w = warp; w < nwords; w += kPartWarps) {
+    const int nwarps = blockDim.x >> 5;
+    for (int w = warp; w < nwords; w += nwarps) {
         const int n0 = start + (w << 5);
         uint32_t mybit = 0;
+        // The loads of up to 4 groups of tokens are issued before any of them is reduced, so a
+        // warp keeps several kilobytes in flight (one 16-byte chunk per lane and tensor and group).
+        constexpr int G = L < 4 ? L : 4;
 #pragma unroll
-        for (int s = 0; s < L; ++s) {
-            const int tok = n0 + s * TPI + lane / L;
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f;      // cosine: dot, |x0|^2, |ref|^2 ; l2: a0 only
-            if (tok < N) {
-                const size_t row = (req + tok) * (size_t)C;
-                for (int ch = sub; ch < chunks; ch += L) {
-                    const uint4 xv = ld_stream128(x_t + row + (ch << 3));
-                    const uint4 vv = ld_stream128(v + row + (ch << 3));
-                    const uint4 rv = ld_stream128(ref + row + (ch << 3));
-                    const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
-                    const uint32_t vs[4] = {vv.x, vv.y, vv.z, vv.w};
-                    const uint32_t rs[4] = {rv.x, rv.y, rv.z, rv.w};
+        for (int s0 = 0; s0 < L; s0 += G) {
+            uint4 xv[G], vv[G], rv[G];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float h0 = fmaf(-t, bf16_lo(vs[k]), bf16_lo(xs[k]));
-                        const float h1 = fmaf(-t, bf16_hi(vs[k]), bf16_hi(xs[k]));
-                        const float r0 = bf16_lo(rs[k]), r1 = bf16_hi(rs[k]);
-                        if (metric == REGIONE_METRIC_COSINE) {
-                            a0 = fmaf(h0, r0, a0); a0 = fmaf(h1, r1, a0);
-                            a1 = fmaf(h0, h0, a1); a1 = fmaf(h1, h1, a1);
-                            a2 = fmaf(r0, r0, a2); a2 = fmaf(r1, r1, a2);
-                        } else {
-                            const float d0 = h0 - r0, d1 = h1 - r1;
-                            a0 = fmaf(d0, d0, a0); a0 = fmaf(d1, d1, a0);
-                        }
-                    }
+            for (int g = 0; g < G; ++g) {
+                const int tok = n0 + (s0 + g) * TPI + lane / L;
+                xv[g] = vv[g] = rv[g] = make_uint4(0, 0, 0, 0);
+                if (tok < N && sub < chunks) {
+                    const size_t at = (req + tok) * (size_t)C + (sub << 3);
+                    xv[g] = ld_stream128(x_t + at);
+                    vv[g] = ld_stream128(v + at);
+                    rv[g] = ld_stream128(ref + at);
                 }
             }
 #pragma unroll
-            for (int d = 1; d < L; d <<= 1) {
-                a0 += __shfl_xor_sync(0xffffffffu, a0, d);
-                a1 += __shfl_xor_sync(0xffffffffu, a1, d);
-                a2 += __shfl_xor_sync(0xffffffffu, a2, d);
+            for (int g = 0; g < G; ++g) {
+                const int s = s0 + g;
+                const int tok = n0 + s * TPI + lane / L;
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f;  // cosine: dot, |x0|^2, |ref|^2 ; l2: a0 only
+                accumulate_chunk(xv[g], vv[g], rv[g], t, metric, a0, a1, a2);
+                if (L == 32 && tok < N) {            // rows wider than 256 channels: further chunks
+                    const size_t row = (req + tok) * (size_t)C;
+                    for (int ch = sub + 32; ch < chunks; ch += 32)
+                        accumulate_chunk(ld_stream128(x_t + row + (ch << 3)),
+                                         ld_stream128(v + row + (ch << 3)),
+                                         ld_stream128(ref + row + (ch << 3)), t, metric, a0, a1, a2);
+                }
+#pragma unroll
+                for (int d = 1; d < L; d <<= 1) {
+                    a0 += __shfl_xor_sync(0xffffffffu, a0, d);
+                    a1 += __shfl_xor_sync(0xffffffffu, a1, d);
+                    a2 += __shfl_xor_sync(0xffffffffu, a2, d);
+                }
+                float sc;
+                bool edited;
+                if (metric == REGIONE_METRIC_COSINE) {
+                    sc = a0 / fmaxf(sqrtf(a1) * sqrtf(a2), 1e-12f);
+                    edited = sc <= threshold;
+                } else {
+                    sc = sqrtf(a0);
+                    edited = sc > threshold;
+                }
+                const bool leader = (sub == 0) && (tok < N);
+                if (leader && score != nullptr) score[req + tok] = sc;
+                const uint32_t ballot = __ballot_sync(0xffffffffu, leader && edited);
+                if (lane / TPI == s) mybit = (ballot >> ((lane % TPI) * L)) & 1u;
             }
-            float sc;
-            bool edited;
-            if (metric == REGIONE_METRIC_COSINE) {
-                sc = a0 / fmaxf(sqrtf(a1) * sqrtf(a2), 1e-12f);
-                edited = sc <= threshold;
-            } else {
-                sc = sqrtf(a0);
-                edited = sc > threshold;
-            }
-            const bool leader = (sub == 0) && (tok < N);
-            if (leader && score != nullptr) score[req + tok] = sc;
-            const uint32_t ballot = __ballot_sync(0xffffffffu, leader && edited);
-            if (lane / TPI == s) mybit = (ballot >> ((lane % TPI) * L)) & 1u;
         }
         const uint32_t word = __ballot_sync(0xffffffffu, mybit != 0);
         if (lane == 0) bits[w] = word;
@@ -290,8 +315,12 @@ static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st
                                     int32_t* edit_idx, int32_t* keep_idx, int32_t* slot,
                                     int32_t* n_edit, float* score) {
     cudaLaunchConfig_t cfg = {};
+    // enough warps per CTA to keep the loads of a large share in flight (a cluster is at most 8
+    // CTAs, so a long request cannot get its memory parallelism from the grid); 512 threads let
+    // two CTAs share an SM, which measured faster than one CTA of 1024
+    const int threads = share >= 2048 ? 512 : 256;
     cfg.gridDim = dim3(csize, B, 1);
-    cfg.blockDim = dim3(kPartThreads, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)(share >> 5) * 8;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
