@@ -180,6 +180,60 @@ def run_reference(args):
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 
+def hbm_sweep(torch, binding, step, d, flush_l2, peak_gbs, iters=10):
+    """Achieved GB/s (algorithmic bytes / CUDA-event time, untimed L2 flush before each launch) of the
+    memory-bound kernels on instances large enough for the figure to mean HBM bandwidth: the cache
+    store and a 6 KB-row gather at the bench workload's size, and partition / velocity decay / merge
+    at 2^21 tokens of 16 channels (32 requests of 65536 tokens)."""
+    bf, i32 = torch.bfloat16, torch.int32
+    out = []
+
+    def timed(name, nbytes, fn):
+        for _ in range(2):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e-3)
+        sec = float(np.median(ts))
+        out.append(dict(kernel=name, mbytes=round(nbytes / 1e6, 1), us=round(sec * 1e6, 1),
+                        gbs=round(nbytes / sec / 1e9, 0), frac_of_measured=round(nbytes / sec / 1e9 / peak_gbs, 3)))
+
+    s = step.shp
+    row = s.H * s.D * 2
+    n_cache = int(step.n_cache.sum().item())
+    timed("rikv_store (bench workload)", n_cache * (4 * row + 4),
+          lambda: binding.rikv_store(d["k"], d["vv"], step.cache_rows, step.n_cache, step.k_cache, step.v_cache))
+    rows = 16384                                            # 100 MB read + 100 MB written
+    idx = (torch.arange(rows, device="cuda", dtype=i32) * 7 % d["k"].shape[1]).sort()[0].to(i32).reshape(1, rows)
+    idx = idx.expand(d["k"].shape[0], rows).contiguous()
+    n_rows = torch.full((d["k"].shape[0],), rows, dtype=i32, device="cuda")
+    dst = torch.empty((d["k"].shape[0], rows, s.H, s.D), dtype=bf, device="cuda")
+    timed("gather of 16384 rows of 6 KB", d["k"].shape[0] * rows * (2 * row + 4),
+          lambda: binding.gather(d["k"], idx, n_rows, dst))
+    B, N, C = 32, 65536, 16
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    x_t, v, ref = ((torch.randn((B, N, C), device="cuda", generator=g)).to(bf) for _ in range(3))
+    mask = torch.empty((B, N), dtype=torch.uint8, device="cuda")
+    e, k, sl = (torch.empty((B, N), dtype=i32, device="cuda") for _ in range(3))
+    ne = torch.empty(B, dtype=i32, device="cuda")
+    timed("partition, 2^21 tokens", B * N * (3 * C * 2 + 9),
+          lambda: binding.partition(x_t, v, ref, 0.7, binding.METRIC_COSINE, 0.1, mask, e, k, sl, ne))
+    n_e = int(ne.sum().item())
+    x_e = torch.zeros((B, N, C), dtype=bf, device="cuda"); v_e = torch.zeros_like(x_e); v_c = torch.zeros_like(x_e)
+    timed("velocity_decay with cache refresh", n_e * 4 * C * 2,
+          lambda: binding.velocity_decay(v_e, 1.0, 1.0 / 28, x_e, ne, v_cache_out=v_c))
+    timed("velocity_decay reusing the cache", n_e * 3 * C * 2,
+          lambda: binding.velocity_decay(v_e, 0.9, 1.0 / 28, x_e, ne))
+    x_out = torch.empty_like(x_t)
+    timed("merge", (B * N - n_e) * (3 * C * 2 + 4) + n_e * (2 * C * 2 + 4),
+          lambda: binding.merge(x_t, v, x_e, sl, 5.0 / 28, x_out))
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -225,6 +279,13 @@ def run_ours(args):
                      metric, wl.threshold)
     step = RegionStep(shp)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
+    drain = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def flush_l2():
+        """Writes 256 MiB (evicts everything), then reads another 256 MiB so that the dirty lines of
+        that write are back in HBM before the timed work starts: L2 is cold and clean."""
+        flush.zero_()
+        drain.view(torch.int32).max()
 
     def one():
         step.run(d["x_t"], d["v"], d["ref"], d["q"], d["k"], d["vv"], t, scale, dt, dt_u)
@@ -248,7 +309,7 @@ def run_ours(args):
     sampler.start()
     wall0 = time.perf_counter()
     for i in range(steps):
-        flush.zero_()
+        flush_l2()
         step.attention_events = aev[i]
         ev[i][0].record()
         one()
@@ -308,6 +369,9 @@ def run_ours(args):
         return
 
     peaks = measured_peaks()
+    hbm_kernels = None
+    if world == 1 and not args.no_hbm_sweep:
+        hbm_kernels = hbm_sweep(torch, binding, step, d, flush_l2, peaks["hbm_gbs"])
     attn_us = float(np.mean(attn_ms) * 1e3)
     achieved = flops / (attn_us * 1e-6) / 1e12
     roofline = dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
@@ -330,12 +394,13 @@ def run_ours(args):
                 config=dict(workload=f"config {cfg}: {wl.name}", batch=wl.batch, image_tokens=wl.n_img,
                             reference_tokens=wl.n_ref, text_tokens=wl.n_text, heads=wl.heads,
                             head_dim=wl.head_dim, n_q=int(n_q[0]), n_kv=int(n_kv[0]),
-                            cache_policy="L2 flushed (256 MiB memset) before every timed step",
+                            cache_policy="L2 flushed before every timed step (256 MiB written, then 256 MiB read to drain the dirty lines)",
                             parallelism=f"replicas x{world} (independent requests, no collective)"),
                 clocks=clocks,
                 e2e=dict(value=e2e_val, unit=UNIT, h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=int(d2h),
                          steps=e2e_steps, ms_per_step=e2e_ms / e2e_steps),
                 gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu_baseline,
+                hbm_kernels=hbm_kernels,
                 step_us=dict(mean=float(step_ms.mean() * 1e3), min=float(step_ms.min() * 1e3),
                              median=float(np.median(step_ms) * 1e3)),
                 attention_us=dict(mean=attn_us, min=float(attn_ms.min() * 1e3)),
@@ -353,6 +418,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 5])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-hbm-sweep", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
