@@ -30,16 +30,22 @@
 // masked in the softmax and their V rows zeroed in shared memory, so garbage
 // (even NaN) behind the live prefix cannot leak.
 //
-// Occupancy: the key tiles of one (request, head, query pair) can be split over
-// several CTAs (split-KV).  Each split then writes its unnormalised output and
-// its (max, sum) pair to the caller's workspace and a small second kernel
-// merges the splits.  The split count is chosen on the host from the
-// capacities so that the grid fills the SMs.
+// Scheduling: the kernel is persistent, one CTA per SM.  A "step" is one key tile of one
+// (request, head, query pair) item; all steps of the launch form one sequence, item after item,
+// which is cut into equal contiguous shares, one per CTA (a stream-K decomposition: the grid is
+// always one balanced wave, whatever the number of items).  A CTA's share is a few segments,
+// each a run of key tiles of one item.  A segment that covers its item completely writes the
+// output rows directly; otherwise it writes its unnormalised output and (max, sum) pair to a
+// slot of the caller's workspace and a small second kernel merges the slots of such items.  The
+// share length is bounded below so that no item is spread over more slots than the workspace
+// holds.  Counts live in device memory, so every CTA derives the same plan from them.
 //
 // Every wait is bounded: if a barrier does not complete within ~2 s the CTA
 // records REGIONE_DEV_TIMEOUT, all roles leave their loops, tensor memory is
 // released and the kernel ends normally.
 #include <cuda.h>
+
+#include <algorithm>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -78,15 +84,109 @@ struct AttnParams {
     const int32_t* n_q;
     const int32_t* n_fresh;
     const int32_t* n_cache;
-    int Nq_cap, Nf_cap, Nc_cap, H;
+    int B, Nq_cap, Nf_cap, Nc_cap, H;
+    int P_cap;           // query pairs per (request, head) at capacity
+    int max_slots;       // workspace slots per item (>= 2)
     float scale_log2e;
     uint16_t* out;
     int32_t* dev_status;
-    int n_splits;        // CTAs sharing the key tiles of one (request, head, query pair)
-    int Nq_pad;          // Nq_cap rounded up to a whole query pair (row pitch of the partials)
-    float* part_o;       // [B, n_splits, Nq_pad, H, D] unnormalised outputs (n_splits > 1)
-    float2* part_ml;     // [B, n_splits, Nq_pad, H]    (running max in the exp2 domain, sum)
+    float* part_o;       // [B, H, P_cap, max_slots, 256, D] unnormalised outputs
+    float2* part_ml;     // [B, H, P_cap, max_slots, 256]    (running max in the exp2 domain, sum)
 };
+
+// ---- the plan every CTA (and the merge kernel) derives from the device-side counts ------------
+struct ReqShape {
+    int nq, nf, nc;      // clamped counts
+    int np;              // live query pairs
+    int nt_c, nt;        // cached key tiles, all key tiles
+    long long items;     // H * np
+};
+
+__device__ __forceinline__ ReqShape req_shape(const AttnParams& p, int b, bool* bad = nullptr) {
+    ReqShape r;
+    int nq = p.n_q[b], nf = p.n_fresh[b], nc = p.n_cache[b];
+    if (nq < 0 || nq > p.Nq_cap || nf < 0 || nf > p.Nf_cap || nc < 0 || nc > p.Nc_cap) {
+        if (bad) *bad = true;
+        nq = max(0, min(nq, p.Nq_cap));
+        nf = max(0, min(nf, p.Nf_cap));
+        nc = max(0, min(nc, p.Nc_cap));
+    }
+    r.nq = nq; r.nf = nf; r.nc = nc;
+    r.np = (nq + 2 * kBM - 1) / (2 * kBM);
+    r.nt_c = (nc + kBN - 1) / kBN;
+    r.nt = r.nt_c + (nf + kBN - 1) / kBN;
+    r.items = (long long)p.H * r.np;
+    return r;
+}
+
+// How the launch's work is cut into one contiguous share per CTA.
+//  - whole items: when handing out whole items wastes at most 6 % of the grid's last round, each
+//    item counts as one step and is never split (no workspace traffic, no merge).
+//  - otherwise a step is one key tile of an item (an item without keys still takes one step: it
+//    writes zeros) and shares may cut items; the share length is then at least
+//    ceil(longest item / (max_slots - 1)) so that an item never spans more than max_slots shares.
+struct Plan {
+    bool whole_items;
+    long long total, chunk;
+    __device__ __forceinline__ int item_len(const ReqShape& r) const {
+        return whole_items ? 1 : max(r.nt, 1);
+    }
+};
+
+__device__ __forceinline__ Plan plan_shares(const AttnParams& p, int grid, bool* bad = nullptr) {
+    Plan pl;
+    long long items = 0, steps = 0;
+    int nt_max = 1;
+    for (int b = 0; b < p.B; ++b) {
+        const ReqShape r = req_shape(p, b, bad);
+        items += r.items;
+        steps += r.items * max(r.nt, 1);
+        if (r.np > 0) nt_max = max(nt_max, r.nt);
+    }
+    const long long per = (items + grid - 1) / grid;
+    pl.whole_items = per * grid * 100 <= items * 106;
+    if (pl.whole_items) {
+        pl.total = items;
+        pl.chunk = max(per, 1LL);
+    } else {
+        pl.total = steps;
+        pl.chunk = (steps + grid - 1) / grid;
+        const long long floor_len = (nt_max + p.max_slots - 2) / (p.max_slots - 1);
+        if (pl.chunk < floor_len) pl.chunk = floor_len;
+        if (pl.chunk < 1) pl.chunk = 1;
+    }
+    return pl;
+}
+
+// The item that step `pos` belongs to.
+struct ItemAt {
+    int b, h, qp;
+    int j0;              // position of `pos` inside the item
+    int len;             // steps of the item
+    long long first;     // first step of the item in the sequence
+    ReqShape r;
+};
+
+__device__ __forceinline__ ItemAt item_at(const AttnParams& p, const Plan& pl, long long pos) {
+    ItemAt it;
+    long long base = 0;
+    int b = 0;
+    ReqShape r = req_shape(p, 0);
+    while (pos >= base + r.items * pl.item_len(r) && b + 1 < p.B) {
+        base += r.items * pl.item_len(r);
+        ++b;
+        r = req_shape(p, b);
+    }
+    it.b = b; it.r = r;
+    it.len = pl.item_len(r);
+    const long long rel = pos - base;
+    const long long item = rel / it.len;
+    it.j0 = (int)(rel - item * it.len);
+    it.h = (int)(item / r.np);
+    it.qp = (int)(item - (long long)it.h * r.np);
+    it.first = base + item * it.len;
+    return it;
+}
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                          int32_t* dev_status) {
@@ -136,45 +236,41 @@ __device__ __forceinline__ float chunk_probabilities(uint32_t tP, const uint32_t
     return (sum[0] + sum[1]) + (sum[2] + sum[3]);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kAttnThreads, 1)
-region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
-                           const __grid_constant__ CUtensorMap tm_kf,
-                           const __grid_constant__ CUtensorMap tm_vf,
-                           const __grid_constant__ CUtensorMap tm_kc,
-                           const __grid_constant__ CUtensorMap tm_vc, const AttnParams p) {
+// The segments of one CTA's share, for one of the two kinds of warpgroup: the softmax warpgroups
+// (SOFTMAX_WG, many registers) or the producer / issuer warpgroup (few).  The two instantiations
+// are called from the two sides of the setmaxnreg split so that each is compiled for its own
+// register budget; both execute the same sequence of CTA-wide barriers.
+template <int D, bool SOFTMAX_WG>
+__device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtensorMap* tm_kf_,
+                                          const CUtensorMap* tm_vf_, const CUtensorMap* tm_kc_,
+                                          const CUtensorMap* tm_vc_, const AttnParams& p,
+                                          long long pos, const long long hi, const Plan pl,
+                                          AttnCtrl* ctrl, uint8_t* smem_gen, const uint32_t sQ,
+                                          const uint32_t sKV, const int warp, const int lane) {
     using Cfg = AttnCfg<D>;
     constexpr int kStages = Cfg::kStages;
     constexpr int kTileBytes = Cfg::kTileBytes;
-
-    const int b = blockIdx.z, h = blockIdx.y;
-    const int split = blockIdx.x % p.n_splits;
-    const int q0 = (blockIdx.x / p.n_splits) * (2 * kBM);
-    int nq = p.n_q[b], nf = p.n_fresh[b], nc = p.n_cache[b];
-    if (nq < 0 || nq > p.Nq_cap || nf < 0 || nf > p.Nf_cap || nc < 0 || nc > p.Nc_cap) {
-        if (threadIdx.x == 0) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
-        nq = max(0, min(nq, p.Nq_cap));
-        nf = max(0, min(nf, p.Nf_cap));
-        nc = max(0, min(nc, p.Nc_cap));
-    }
-    if (q0 >= nq) return;                               // uniform for the CTA
-    const int ntq = (nq - q0 > kBM) ? 2 : 1;            // live query tiles of this CTA
-    const int nt_c = (nc + kBN - 1) / kBN;
-    const int nt_f = (nf + kBN - 1) / kBN;
-    const int n_tiles_all = nt_c + nt_f;
-    // this CTA's share of the key tiles: [j_first, j_first + n_tiles)
-    const int j_first = (int)(((long long)split * n_tiles_all) / p.n_splits);
-    const int n_tiles = (int)(((long long)(split + 1) * n_tiles_all) / p.n_splits) - j_first;
-
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
-    const uint32_t sQ = smem_base;                      // 2 query tiles
-    const uint32_t sKV = smem_base + 2 * kTileBytes;    // ring of K/V stages
-    AttnCtrl* ctrl = reinterpret_cast<AttnCtrl*>(smem_gen + Cfg::kSmemTiles);
     volatile int* abort_flag = &ctrl->abort_flag;
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const CUtensorMap& tm_q = *tm_q_;
+    const CUtensorMap& tm_kf = *tm_kf_;
+    const CUtensorMap& tm_vf = *tm_vf_;
+    const CUtensorMap& tm_kc = *tm_kc_;
+    const CUtensorMap& tm_vc = *tm_vc_;
+    while (pos < hi) {
+    // ---- the segment: key tiles [j_first, j_first + n_tiles) of item (b, h, query pair) ----
+    const ItemAt it = item_at(p, pl, pos);
+    const int seg_len = (int)min((long long)(it.len - it.j0), hi - pos);
+    const int b = it.b, h = it.h;
+    const int q0 = it.qp * (2 * kBM);
+    const int nq = it.r.nq, nf = it.r.nf, nc = it.r.nc, nt_c = it.r.nt_c;
+    const int ntq = (nq - q0 > kBM) ? 2 : 1;            // live query tiles of this segment
+    const int j_first = it.j0;
+    const int n_tiles = pl.whole_items ? it.r.nt : (it.r.nt == 0 ? 0 : seg_len);
+    // slot of this segment among the shares that touch the item; a lone segment writes the output
+    const int c_first = (int)(it.first / pl.chunk);
+    const int n_slots = pl.whole_items ? 1 : (int)((it.first + it.len - 1) / pl.chunk) - c_first + 1;
+    const int slot = (int)blockIdx.x - c_first;
+    const bool direct = n_slots == 1;
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(ptx::smem_addr(&ctrl->q_full), 1);
@@ -189,20 +285,15 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
             ptx::mbar_init(ptx::smem_addr(&ctrl->o_final[t]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctrl->turn[t]), kBM / 32);
         }
-        ctrl->abort_flag = 0;
         ptx::fence_barrier_init();
-    }
-    if (warp == 9) {
-        ptx::tmem_alloc(ptx::smem_addr(&ctrl->tmem_base), 512);
-        ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem = ctrl->tmem_base;
 
-    // key tile jl of this CTA -> (segment, first row, live rows); a tile yields one P chunk when
-    // at most 64 of its keys are live, else two
+    // key tile jl of this segment -> (segment of the KV sequence, first row, live rows); a tile
+    // yields one P chunk when at most 64 of its keys are live, else two
     auto tile_seg = [&](int jl, bool& cached, int& row0, int& valid) {
         const int j = j_first + jl;
         cached = j < nt_c;
@@ -216,10 +307,10 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         return valid > kBH ? 2 : 1;
     };
 
-    if (warp >= 8) ptx::reg_dealloc<56>();              // producer / issuer warpgroup gives registers up
+    if constexpr (!SOFTMAX_WG) {
     if (warp == 8) {
         // ================= TMA producer =================
-        if (lane == 0) {
+        if (lane == 0 && n_tiles > 0) {
             ptx::prefetch_tensormap(&tm_q);
             ptx::prefetch_tensormap(j_first < nt_c ? &tm_kc : &tm_kf);
             ptx::prefetch_tensormap(j_first < nt_c ? &tm_vc : &tm_vf);
@@ -251,7 +342,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         // ================= MMA issuers: warp 9 for query tile 0, warp 10 for query tile 1 ========
         // Each whole warp walks its loop and waits on the barriers; one elected lane issues.
         const int t = warp - 9;
-        if (t < ntq) {
+        if (t < ntq && n_tiles > 0) {
             constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
             constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
@@ -334,9 +425,9 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                 __syncwarp();
             }
         }
+    }
     } else if (warp < 4 * ntq) {
         // ================= softmax / correction / epilogue =================
-        ptx::reg_alloc<224>();                              // a row of 128 logits stays in registers
         const int t = warp >> 2;
         const int row = ((warp & 3) << 5) + lane;                  // row of the query tile
         const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
@@ -440,7 +531,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
             ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status);
             if (ok) ptx::tc_fence_after_sync();
         }
-        if (p.n_splits == 1) {
+        if (direct) {
             // O / l -> bf16 -> out
             uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D;
             if (n_tiles == 0) {
@@ -468,8 +559,9 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                 }
             }
         } else {
-            // unnormalised O and (m, l) of this split -> workspace; a split without keys has l = 0
-            const size_t prow = (((size_t)b * p.n_splits + split) * p.Nq_pad + qrow) * p.H + h;
+            // unnormalised O and (m, l) of this segment -> its workspace slot
+            const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + it.qp;
+            const size_t prow = (item_idx * p.max_slots + slot) * (2 * kBM) + t * kBM + row;
             if (n_tiles == 0) {
                 if (live) p.part_ml[prow] = make_float2(-INFINITY, 0.f);
             } else if (ok) {
@@ -491,6 +583,73 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
     }
 
+    // ---- end of the segment: every role is done with shared and tensor memory ----
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    if (threadIdx.x == 0) {
+        ptx::mbar_inval(ptx::smem_addr(&ctrl->q_full));
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_inval(ptx::smem_addr(&ctrl->kv_full[s]));
+            ptx::mbar_inval(ptx::smem_addr(&ctrl->kv_empty[s]));
+        }
+        for (int t = 0; t < 2; ++t) {
+            ptx::mbar_inval(ptx::smem_addr(&ctrl->s_full[t]));
+            ptx::mbar_inval(ptx::smem_addr(&ctrl->p_full[t][0]));
+            ptx::mbar_inval(ptx::smem_addr(&ctrl->p_full[t][1]));
+            ptx::mbar_inval(ptx::smem_addr(&ctrl->o_final[t]));
+            ptx::mbar_inval(ptx::smem_addr(&ctrl->turn[t]));
+        }
+    }
+    pos += pl.whole_items ? (long long)gridDim.x : (long long)seg_len;
+    if (*abort_flag) break;
+    }   // segments
+}
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
+                           const __grid_constant__ CUtensorMap tm_kf,
+                           const __grid_constant__ CUtensorMap tm_vf,
+                           const __grid_constant__ CUtensorMap tm_kc,
+                           const __grid_constant__ CUtensorMap tm_vc, const AttnParams p) {
+    using Cfg = AttnCfg<D>;
+    constexpr int kTileBytes = Cfg::kTileBytes;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
+    const uint32_t sQ = smem_base;                      // 2 query tiles
+    const uint32_t sKV = smem_base + 2 * kTileBytes;    // ring of K/V stages
+    AttnCtrl* ctrl = reinterpret_cast<AttnCtrl*>(smem_gen + Cfg::kSmemTiles);
+    volatile int* abort_flag = &ctrl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // this CTA's share [pos, hi) of the step sequence
+    bool bad = false;
+    const Plan pl = plan_shares(p, gridDim.x, &bad);
+    if (bad && blockIdx.x == 0 && threadIdx.x == 0) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+    // (whole items are dealt round-robin, so that the CTAs running at any one time work on
+    // neighbouring items, which share K/V tiles in L2; a share of steps is one contiguous range)
+    long long pos = pl.whole_items ? (long long)blockIdx.x : (long long)blockIdx.x * pl.chunk;
+    const long long hi = pl.whole_items ? pl.total : min(pos + pl.chunk, pl.total);
+    if (pos >= hi) return;                              // uniform for the CTA
+
+    if (threadIdx.x == 0) ctrl->abort_flag = 0;
+    if (warp == 9) {
+        ptx::tmem_alloc(ptx::smem_addr(&ctrl->tmem_base), 512);
+        ptx::tmem_relinquish();
+    }
+    if (warp >= 8) {
+        ptx::reg_dealloc<56>();                         // producer / issuer warpgroup gives registers up
+        run_share<D, false>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
+                            sKV, warp, lane);
+    } else {
+        ptx::reg_alloc<224>();                          // a row of 128 logits stays in registers
+        run_share<D, true>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
+                           sKV, warp, lane);
+    }
+
     // ================= teardown =================
     if (*abort_flag) {
         // give copies and MMAs that are still in flight time to land before tensor memory and
@@ -502,45 +661,60 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     __syncthreads();
     if (warp == 9) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem, 512);
+        ptx::tmem_dealloc(ctrl->tmem_base, 512);
     }
 }
 
-// Merges the splits of one output row: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
-// One warp per (request, query row, head); a lane owns D / 32 consecutive columns.
+// Merges the workspace slots of the items that were spread over several shares:
+// out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  One warp per (request, query row, head); a
+// lane owns D / 32 consecutive columns.  `grid_main` is the grid of the attention kernel, from which
+// the same plan (share length, slots per item) is derived.
 template <int D>
 __global__ void __launch_bounds__(256)
-region_attention_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml,
-                                const int32_t* __restrict__ n_q, int Nq_cap, int Nq_pad, int H,
-                                int n_splits, uint16_t* __restrict__ out) {
+region_attention_combine_kernel(const AttnParams p, int grid_main) {
     const int b = blockIdx.z;
     const int lane = threadIdx.x & 31;
     const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);     // (row, head) pair
-    const int qrow = (int)(w / H), h = (int)(w % H);
-    const int nq = max(0, min(n_q[b], Nq_cap));
-    if (qrow >= nq) return;
+    const int qrow = (int)(w / p.H), h = (int)(w % p.H);
+    const ReqShape r = req_shape(p, b);
+    if (qrow >= r.nq) return;
+    const Plan pl = plan_shares(p, grid_main);
+    if (pl.whole_items) return;                      // nothing was split
+    long long base = 0;
+    for (int bb = 0; bb < b; ++bb) {
+        const ReqShape rb = req_shape(p, bb);
+        base += rb.items * pl.item_len(rb);
+    }
+    const int qp = qrow / (2 * kBM);
+    const int len = pl.item_len(r);
+    const long long first = base + ((long long)h * r.np + qp) * len;
+    const int c_first = (int)(first / pl.chunk);
+    const int n_slots = (int)((first + len - 1) / pl.chunk) - c_first + 1;
+    if (n_slots == 1) return;                        // written directly by the attention kernel
+    const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + qp;
+    const size_t prow0 = item_idx * p.max_slots * (2 * kBM) + (qrow - qp * 2 * kBM);
     constexpr int E = D / 32;
     float M = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) {
-        const float2 ml = part_ml[(((size_t)b * n_splits + s) * Nq_pad + qrow) * H + h];
+    for (int s = 0; s < n_slots; ++s) {
+        const float2 ml = p.part_ml[prow0 + (size_t)s * (2 * kBM)];
         if (ml.y > 0.f) M = fmaxf(M, ml.x);
     }
     float acc[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
     float L = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const size_t prow = (((size_t)b * n_splits + s) * Nq_pad + qrow) * H + h;
-        const float2 ml = part_ml[prow];
+    for (int s = 0; s < n_slots; ++s) {
+        const size_t prow = prow0 + (size_t)s * (2 * kBM);
+        const float2 ml = p.part_ml[prow];
         if (!(ml.y > 0.f)) continue;
         const float wgt = fast_exp2(ml.x - M);
         L = fmaf(wgt, ml.y, L);
-        const float* po = part_o + prow * D + lane * E;
+        const float* po = p.part_o + prow * D + lane * E;
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[e] = fmaf(wgt, po[e], acc[e]);
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
-    uint16_t* orow = out + (((size_t)b * Nq_cap + qrow) * H + h) * D + lane * E;
+    uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D + lane * E;
 #pragma unroll
     for (int e = 0; e < E; e += 2)
         *reinterpret_cast<uint32_t*>(orow + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
@@ -561,24 +735,22 @@ static int sm_count() {
     return n;
 }
 
-// Split count from the capacities alone (so the workspace query and the launch agree): the
-// smallest count, at most 8 and leaving at least 4 key tiles per split, whose grid wastes the
-// least of its last wave.
-static int choose_splits(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H) {
-    const long long items = (long long)((Nq_cap + 2 * kBM - 1) / (2 * kBM)) * H * B;
-    const int tiles = (Nf_cap + kBN - 1) / kBN + (Nc_cap + kBN - 1) / kBN;
-    const int sms = sm_count();
-    int best = 1;
-    double best_eff = 0.0;
-    for (int s = 1; s <= 8 && (s == 1 || tiles / s >= 4); ++s) {
-        const long long ctas = items * s;
-        const double eff = (double)ctas / (double)(((ctas + sms - 1) / sms) * sms);
-        if (eff > best_eff + 0.02) {
-            best_eff = eff;
-            best = s;
-        }
-    }
-    return best;
+// Launch shape from the capacities alone (so the workspace query and the launch agree): a
+// persistent grid of one CTA per SM (fewer if there are fewer steps), and enough workspace slots
+// per item that the longest item can be spread over the shares it meets at that grid size.
+struct LaunchPlan {
+    int grid, P_cap, max_slots;
+};
+
+static LaunchPlan plan_launch(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H) {
+    LaunchPlan lp;
+    lp.P_cap = (Nq_cap + 2 * kBM - 1) / (2 * kBM);
+    const long long nt_cap = std::max(1, (Nf_cap + kBN - 1) / kBN + (Nc_cap + kBN - 1) / kBN);
+    const long long total_cap = (long long)B * H * lp.P_cap * nt_cap;
+    lp.grid = (int)std::min<long long>(sm_count(), std::max<long long>(total_cap, 1));
+    const long long share = (total_cap + lp.grid - 1) / lp.grid;
+    lp.max_slots = (int)std::min<long long>(8, std::max<long long>(2, (nt_cap + share - 1) / share + 1));
+    return lp;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -614,17 +786,18 @@ static bool make_map(CUtensorMap* map, const void* base, int B, int rows, int H,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static inline int pad_rows(int Nq_cap) { return (Nq_cap + 2 * kBM - 1) / (2 * kBM) * (2 * kBM); }
+static inline size_t slot_rows(const LaunchPlan& lp, int B, int H) {
+    return (size_t)B * H * lp.P_cap * lp.max_slots * (2 * kBM);
+}
 
 size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D) {
-    const int s = choose_splits(B, Nq_cap, Nf_cap, Nc_cap, H);
-    if (s == 1) return 0;
-    const size_t rows = (size_t)B * s * pad_rows(Nq_cap) * H;
+    const LaunchPlan lp = plan_launch(B, Nq_cap, Nf_cap, Nc_cap, H);
+    const size_t rows = slot_rows(lp, B, H);
     return ((rows * D * sizeof(float) + 255) & ~(size_t)255) + rows * sizeof(float2);
 }
 
 template <int D>
-static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int B, cudaStream_t st) {
+static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, cudaStream_t st) {
     using Cfg = AttnCfg<D>;
     static bool configured = false;
     if (!configured) {
@@ -634,16 +807,12 @@ static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int B, cuda
             return REGIONE_CUDA_ERROR;
         configured = true;
     }
-    dim3 grid((prm.Nq_cap + 2 * kBM - 1) / (2 * kBM) * prm.n_splits, prm.H, B);
     region_attention_tc_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, st>>>(
         maps[0], maps[1], maps[2], maps[3], maps[4], prm);
     if (cudaGetLastError() != cudaSuccess) return REGIONE_CUDA_ERROR;
-    if (prm.n_splits > 1) {
-        const long long warps = (long long)prm.Nq_cap * prm.H;
-        dim3 cgrid((unsigned)((warps + 7) / 8), 1, B);
-        region_attention_combine_kernel<D><<<cgrid, 256, 0, st>>>(
-            prm.part_o, prm.part_ml, prm.n_q, prm.Nq_cap, prm.Nq_pad, prm.H, prm.n_splits, prm.out);
-    }
+    const long long warps = (long long)prm.Nq_cap * prm.H;
+    dim3 cgrid((unsigned)((warps + 7) / 8), 1, prm.B);
+    region_attention_combine_kernel<D><<<cgrid, 256, 0, st>>>(prm, grid);
     return launch_status(cudaGetLastError());
 }
 
@@ -664,21 +833,18 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
         !make_map(&maps[2], vf, B, Nf_cap, H, D) || !make_map(&maps[3], kc, B, Nc_cap, H, D) ||
         !make_map(&maps[4], vc, B, Nc_cap, H, D))
         return REGIONE_CUDA_ERROR;
+    const LaunchPlan lp = plan_launch(B, Nq_cap, Nf_cap, Nc_cap, H);
     AttnParams prm;
     prm.n_q = n_q; prm.n_fresh = n_fresh; prm.n_cache = n_cache;
-    prm.Nq_cap = Nq_cap; prm.Nf_cap = Nf_cap; prm.Nc_cap = Nc_cap; prm.H = H;
+    prm.B = B; prm.Nq_cap = Nq_cap; prm.Nf_cap = Nf_cap; prm.Nc_cap = Nc_cap; prm.H = H;
+    prm.P_cap = lp.P_cap; prm.max_slots = lp.max_slots;
     prm.scale_log2e = scale * 1.4426950408889634f;
     prm.out = out; prm.dev_status = dev_status;
-    prm.n_splits = choose_splits(B, Nq_cap, Nf_cap, Nc_cap, H);
-    prm.Nq_pad = pad_rows(Nq_cap);
-    prm.part_o = nullptr; prm.part_ml = nullptr;
-    if (prm.n_splits > 1) {
-        const size_t rows = (size_t)B * prm.n_splits * prm.Nq_pad * H;
-        prm.part_o = reinterpret_cast<float*>(workspace);
-        prm.part_ml = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(workspace) +
-                                                ((rows * D * sizeof(float) + 255) & ~(size_t)255));
-    }
-    return D == 64 ? launch_tc<64>(maps, prm, B, st) : launch_tc<128>(maps, prm, B, st);
+    const size_t rows = slot_rows(lp, B, H);
+    prm.part_o = reinterpret_cast<float*>(workspace);
+    prm.part_ml = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(workspace) +
+                                            ((rows * D * sizeof(float) + 255) & ~(size_t)255));
+    return D == 64 ? launch_tc<64>(maps, prm, lp.grid, st) : launch_tc<128>(maps, prm, lp.grid, st);
 }
 
 // ---- variant with library-owned scratch -----------------------------------------------------
