@@ -242,6 +242,42 @@ def hbm_sweep(torch, binding, step, d, flush_l2, peak_gbs, iters=10):
     return out
 
 
+def ratio_sweep(torch, binding, synth, flush_l2, to_dev, steps=20):
+    """Denoise-step time against the edit-mask ratio on the Qwen-Image-Edit-shaped workload (config 3):
+    one region step (all 12 calls) and its attention call per ratio, CUDA events, L2 flushed per step."""
+    from paper_2510_25590_b200.step import RegionStep, StepShapes, plan_capacity
+    wl = synth.WORKLOADS[3]
+    qkv = synth.make_qkv_full(wl)
+    dq, dk, dv = (to_dev(qkv[k]) for k in ("q", "k", "v"))
+    out = []
+    for ratio in wl.ratios:
+        lat = synth.make_latents(wl, ratio)
+        x_t, v, ref = (to_dev(lat[k]) for k in ("x_t", "v", "ref"))
+        cap = plan_capacity(x_t, v, ref, lat["t"], binding.METRIC_COSINE, wl.threshold)
+        step = RegionStep(StepShapes(wl.batch, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads,
+                                     wl.head_dim, cap, binding.METRIC_COSINE, wl.threshold))
+        run = lambda: step.run(x_t, v, ref, dq, dk, dv, lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0)
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+        for i in range(steps):
+            flush_l2()
+            step.attention_events = (ev[i][1], ev[i][2])
+            ev[i][0].record(); run(); ev[i][3].record()
+        torch.cuda.synchronize()
+        step.attention_events = None
+        assert int(step.dev_status[0]) == 0
+        n_q = int(step.n_q[0]); n_kv = n_q + int(step.n_cache[0])
+        st_us = float(np.mean([e[0].elapsed_time(e[3]) for e in ev]) * 1e3)
+        at_us = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]) * 1e3)
+        fl = 4.0 * wl.heads * wl.head_dim * n_q * n_kv
+        out.append(dict(ratio=ratio, n_q=n_q, n_kv=n_kv, step_us=round(st_us, 1), attention_us=round(at_us, 1),
+                        attention_tflops=round(fl / at_us / 1e6, 1)))
+        del step
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -380,6 +416,9 @@ def run_ours(args):
     hbm_kernels = None
     if world == 1 and not args.no_hbm_sweep:
         hbm_kernels = hbm_sweep(torch, binding, step, d, flush_l2, peaks["hbm_gbs"])
+    step_vs_ratio = None
+    if world == 1 and not args.no_ratio_sweep:
+        step_vs_ratio = ratio_sweep(torch, binding, synth, flush_l2, dev)
     attn_us = float(np.mean(attn_ms) * 1e3)
     achieved = flops / (attn_us * 1e-6) / 1e12
     roofline = dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
@@ -408,7 +447,7 @@ def run_ours(args):
                 e2e=dict(value=e2e_val, unit=UNIT, h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=int(d2h),
                          steps=e2e_steps, ms_per_step=e2e_ms / e2e_steps),
                 gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu_baseline,
-                hbm_kernels=hbm_kernels,
+                hbm_kernels=hbm_kernels, denoise_step_us_vs_mask_ratio=step_vs_ratio,
                 step_us=dict(mean=float(step_ms.mean() * 1e3), min=float(step_ms.min() * 1e3),
                              median=float(np.median(step_ms) * 1e3)),
                 attention_us=dict(mean=attn_us, min=float(attn_ms.min() * 1e3)),
@@ -427,6 +466,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 5])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-hbm-sweep", action="store_true")
+    ap.add_argument("--no-ratio-sweep", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
