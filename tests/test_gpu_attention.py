@@ -212,3 +212,41 @@ def test_tensor_core_kernel_agrees_with_cuda_core_kernel_on_every_row():
     assert ma <= 2e-2 and rr <= 5e-3, (ma, rr)
     want = orc.region_attention(c["q"], c["kf"], c["vf"], c["kc"], c["vc"], c["nq"], c["nf"], c["nc"])
     assert_close(s, want, "cuda-core kernel vs oracle")
+
+
+@pytest.mark.parametrize("caps,counts", [
+    # capacities far above the live counts: the plan comes from the device-side counts, the workspace
+    # slot bound from the capacities
+    ((2048, 2048, 8192), [(130, 100, 700)]),
+    # a batch with an empty request, a one-row request and a request without any key
+    ((300, 256, 1024), [(0, 50, 300), (1, 3, 5), (257, 0, 0), (300, 256, 1024)]),
+    # very few queries against a long key sequence: every item is cut into the maximum number of slots
+    ((128, 128, 16384), [(128, 128, 16384)]),
+    # many short items: whole items are dealt round-robin, nothing is split
+    ((256, 128, 256), [(256, 128, 256)] * 6),
+])
+def test_scheduling_plans(caps, counts):
+    cap_q, cap_f, cap_c = caps
+    B, H, D = len(counts), 5, 128
+    rng = np.random.default_rng(cap_q + cap_c + B)
+    q = _rand_bf16(rng, (B, cap_q, H, D), 0.3)
+    kf, vf = _rand_bf16(rng, (B, cap_f, H, D), 0.3), _rand_bf16(rng, (B, cap_f, H, D))
+    kc, vc = _rand_bf16(rng, (B, cap_c, H, D), 0.3), _rand_bf16(rng, (B, cap_c, H, D))
+    n_q = np.array([c[0] for c in counts], np.int32)
+    n_f = np.array([c[1] for c in counts], np.int32)
+    n_c = np.array([c[2] for c in counts], np.int32)
+    got = run_attention(q, kf, vf, kc, vc, n_q, n_f, n_c, poison=float("nan"))
+    samples = []
+    for b in range(B):
+        if n_q[b] == 0:
+            continue
+        rows = sorted(set([0, int(n_q[b]) - 1] + rng.integers(0, n_q[b], 6).tolist()))
+        samples += [(b, r, int(rng.integers(0, H))) for r in rows]
+    live = [(b, r, h) for (b, r, h) in samples if n_f[b] + n_c[b] > 0]
+    want = orc.region_attention_rows(q, kf, vf, kc, vc, n_f, n_c, live)
+    assert_close(np.stack([got[b, r, h] for (b, r, h) in live]), want, f"plan {caps}")
+    for (b, r, h) in samples:
+        if n_f[b] + n_c[b] == 0:
+            assert np.all(got[b, r, h] == 0.0)              # no key at all: the row is zero
+    for b in range(B):
+        assert np.all(got[b, n_q[b]:] == -3.0)              # rows past n_q are not written
