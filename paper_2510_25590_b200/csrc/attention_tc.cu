@@ -56,6 +56,7 @@ constexpr int kAttnThreads = 384;        // 2 softmax warpgroups + 1 of producer
 constexpr int kBM = 128;                 // query rows per tile
 constexpr int kBN = 128;                 // key rows per shared-memory tile
 constexpr int kBH = 64;                  // key rows per P chunk (half a tile)
+constexpr int kPolyEvery = 2;             // every kPolyEvery-th pair computes one of its two exponentials on the FMA pipe
 constexpr int kHalfBytes = 128 * 64 * 2; // one 128-row x 64-column bf16 box (128-byte rows)
 constexpr long long kTimeoutCycles = 4000000000LL;
 
@@ -216,6 +217,20 @@ __device__ __forceinline__ float chunk_max(const uint32_t* s, int valid) {
     return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 }
 
+// 2^x for x <= 0 on the FMA pipe: x = n + f with n = round(x) (the magic-number addition leaves n in
+// the low mantissa bits of t), 2^f by a cubic on [-0.5, 0.5] (relative error 7.5e-5, far below the
+// bf16 rounding of the probabilities), n added to the exponent field.  Used for part of the
+// exponentials so that they do not all queue on the special-function unit.
+__device__ __forceinline__ float poly_exp2(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = x + 12582912.f;
+    const float f = x - (t - 12582912.f);
+    float p = fmaf(f, 0.0551716f, 0.2426111f);
+    p = fmaf(p, f, 0.6932610f);
+    p = fmaf(p, f, 0.9999281f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
 // p = 2^(s*c - m) for 64 logits, written to tensor memory at `tP` (32 columns) as packed bf16;
 // returns their fp32 sum.
 template <bool MASK>
@@ -226,7 +241,8 @@ __device__ __forceinline__ float chunk_probabilities(uint32_t tP, const uint32_t
 #pragma unroll
     for (int i = 0; i < kBH / 2; ++i) {
         float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, -m));
-        float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m));
+        float p1 = (i % kPolyEvery == 0) ? poly_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m))
+                                         : fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m));
         if (MASK && 2 * i >= valid) p0 = 0.f;
         if (MASK && 2 * i + 1 >= valid) p1 = 0.f;
         sum[i & 3] += p0 + p1;
