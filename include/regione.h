@@ -229,6 +229,21 @@ int regione_region_attention_static(const regione_bf16* q,
 int regione_avd_step(double* running_product, double dt, double gamma, double delta, int* reuse);
 
 /*
+ * Fit of the timestep-aware decay correction gamma (Sec. 4, "Adaptive Velocity Decay
+ * Cache", decay-factor equation: ||v_{t_i}|| / ||v_{t_{i+1}}|| = (1 - dt_i) * gamma_{t_i},
+ * gamma "obtained by fitting on a randomly sampled dataset").  From the velocities of S
+ * sampled trajectories at T1 consecutive steps:
+ *     norms[s, i] = || v[s, i, :] ||_2
+ *     gamma[i]    = mean_s( norms[s, i] / norms[s, i+1] ) / (1 - dt[i]),     i < T1 - 1
+ * (index i+1 is the earlier, noisier step).  The paper does not say how it fits; the mean of
+ * the per-sample ratios is this library's reading.
+ * v : dev bf16 [S, T1, n], n a multiple of 8;  dt : dev f32 [T1-1];
+ * norms : dev f32 [S, T1] (output);  gamma : dev f32 [T1-1] (output).
+ */
+int regione_gamma_fit(const regione_bf16* v, int S, int T1, int64_t n, const float* dt,
+                      float* norms, float* gamma, void* stream);
+
+/*
  * Decayed cached velocity and Euler update of the edited tokens (Sec. 4, the
  * case equation of the AVDCache; Sec. 3, the Euler sampler equation):
  *     v_use = scale * v_in[b,j,:]

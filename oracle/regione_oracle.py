@@ -318,6 +318,20 @@ def avd_schedule(timesteps, gammas, delta, first, last):
     return out
 
 
+def gamma_fit(v, dt):
+    """gamma_{t_i} from sampled velocities (decay-factor equation solved for gamma).
+
+    v [S, T1, n] (index i+1 = the earlier step), dt [T1-1].  Per sample the ratio
+    ||v_i|| / ||v_{i+1}||, averaged over the samples, divided by the solver factor (1 - dt_i).
+    The paper only says gamma is fitted on sampled data; the mean of ratios is this reading.
+    Returns (norms [S, T1], gamma [T1-1]).
+    """
+    v = _f64(v)
+    norms = np.sqrt(np.sum(v * v, axis=-1))
+    ratio = norms[:, :-1] / norms[:, 1:]
+    return norms, ratio.mean(axis=0) / (1.0 - _f64(dt))
+
+
 def velocity_decay(v_in, scale, dt, x_e, n_edit):
     """v^E = scale * v_in;  X^E_{t_{j-1}} = X^E_{t_j} - dt * v^E  (Euler sampler equation).
 

@@ -36,6 +36,7 @@ SIGNATURES = {
     "regione_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, c_size_t, _P, _P]),
     "regione_region_attention_static": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, _P]),
     "regione_avd_step": (c_int, [POINTER(c_double), c_double, c_double, c_double, POINTER(c_int)]),
+    "regione_gamma_fit": (c_int, [_P, c_int, c_int, c_int64, _P, _P, _P, _P]),
     "regione_velocity_decay": (c_int, [_P, c_float, c_float, _P, _P, _P, c_int, c_int, c_int, _P, _P]),
     "regione_merge": (c_int, [_P, _P, _P, _P, c_float, c_int, c_int, c_int, c_int, _P, _P, _P]),
 }
@@ -228,6 +229,16 @@ def avd_step(running_product: float, dt: float, gamma: float, delta: float):
     _check(load().regione_avd_step(ctypes.byref(p), dt, gamma, delta, ctypes.byref(r)),
            "regione_avd_step")
     return p.value, bool(r.value)
+
+
+def gamma_fit(v, dt, norms, gamma, stream=None):
+    """v [S, T1, n] bf16, dt [T1-1] f32 -> norms [S, T1], gamma [T1-1] (both f32, written)."""
+    torch = _torch()
+    S, T1, n = v.shape
+    _check(load().regione_gamma_fit(
+        _ptr(v, torch.bfloat16, "v"), S, T1, n, _ptr(dt, torch.float32, "dt"),
+        _ptr(norms, torch.float32, "norms"), _ptr(gamma, torch.float32, "gamma"), _stream(stream)),
+        "regione_gamma_fit")
 
 
 def velocity_decay(v_in, scale, dt, x_e, n_edit, v_cache_out=None, dev_status=None, stream=None):

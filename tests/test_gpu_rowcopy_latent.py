@@ -124,3 +124,19 @@ def test_merge(cfg, grid):
     buf = dev_bf16(lat["x_t"])
     binding.merge(buf, dev_bf16(lat["v"]), dev_bf16(x_e_full), dev_i32(full), dt, buf)
     assert np.array_equal(host_f64(buf), x_e_full)
+
+
+@pytest.mark.parametrize("S,T1,n", [(3, 5, 8), (4, 29, 4096 * 16), (2, 2, 1000 * 8)])
+def test_gamma_fit(S, T1, n):
+    import torch
+    rng = np.random.default_rng(S * 100 + T1)
+    v = synth.bf16_round(rng.standard_normal((S, T1, n)).astype(np.float32) *
+                         np.linspace(1.0, 2.0, T1, dtype=np.float32)[None, :, None])
+    dt = np.full(T1 - 1, 1.0 / 28.0, np.float32)
+    norms = torch.full((S, T1), -1.0, dtype=torch.float32, device="cuda")
+    gamma = torch.full((T1 - 1,), -1.0, dtype=torch.float32, device="cuda")
+    binding.gamma_fit(dev_bf16(v), torch.from_numpy(dt).cuda(), norms, gamma)
+    torch.cuda.synchronize()
+    want_n, want_g = orc.gamma_fit(v, dt)
+    assert np.allclose(norms.cpu().numpy(), want_n, rtol=2e-6)
+    assert np.allclose(gamma.cpu().numpy(), want_g, rtol=1e-5)

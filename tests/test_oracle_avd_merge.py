@@ -93,3 +93,25 @@ def test_stage_schedule_counts():
     assert kinds[:6] == ["full"] * 5 + ["full_store"]
     assert dict(s)[17] == "full_store" and dict(s)[2] == "full_store" and dict(s)[1] == "full"
     assert all(dict(s)[j] == "region" for j in list(range(22, 17, -1)) + list(range(16, 2, -1)))
+
+
+def test_gamma_fit_recovers_planted_corrections_and_reduces_to_one_for_the_residual_cache():
+    # Appendix: under residual caching v_{i} = (1 - dt_i) v_{i+1}, i.e. gamma = 1; a planted extra
+    # factor g_i per step must come back exactly, whatever the direction and scale of the samples
+    rng = np.random.default_rng(3)
+    S, T, n = 5, 7, 64
+    dt = rng.uniform(0.01, 0.1, T)
+    g = rng.uniform(0.9, 1.0, T)
+    v = np.empty((S, T + 1, n))
+    v[:, T] = rng.standard_normal((S, n)) * rng.uniform(0.5, 3.0, (S, 1))
+    for i in range(T - 1, -1, -1):
+        v[:, i] = (1.0 - dt[i]) * g[i] * v[:, i + 1]
+    norms, gamma = orc.gamma_fit(v, dt)
+    assert np.allclose(gamma, g, rtol=1e-12)
+    assert np.allclose(norms[:, 0] / norms[:, T], np.prod((1 - dt) * g), rtol=1e-12)
+    _, gamma1 = orc.gamma_fit(v / g.prod(), dt)                     # a global rescale changes nothing
+    assert np.allclose(gamma1, g, rtol=1e-12)
+    # brute force on one entry
+    i = 3
+    want = np.mean([np.linalg.norm(v[s, i]) / np.linalg.norm(v[s, i + 1]) for s in range(S)]) / (1 - dt[i])
+    assert abs(gamma[i] - want) < 1e-14
