@@ -131,6 +131,17 @@ int regione_gather(const void* src, const int32_t* idx, const int32_t* n, int B,
                    void* dst, int32_t* dev_status, void* stream);
 
 /*
+ * The same gather for up to 4 tensors of identical shape that share one index list, in one
+ * launch (Algorithm 1 gathers X and v, and the recomputed rows of Q, K and V, with the same
+ * E_index): dsts[i][b, j, :] = srcs[i][b, idx[b, j], :].
+ * srcs, dsts : host arrays of n_tensors device pointers (1 <= n_tensors <= 4).
+ */
+int regione_gather_multi(const void* const* srcs, void* const* dsts, int n_tensors,
+                         const int32_t* idx, const int32_t* n, int B, int64_t src_rows,
+                         int64_t idx_stride, int64_t dst_rows_cap, int64_t row_bytes,
+                         int32_t* dev_status, void* stream);
+
+/*
  * Token scatter, the inverse placement (Sec. 4: results are "re-gathered according
  * to their spatial positions"; Algorithm 1, the gather(...) line):
  *     dst[b, idx[b, j], :] = src[b, j, :]     for j < min(n[b], src_rows_cap)

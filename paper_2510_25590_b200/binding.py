@@ -30,6 +30,7 @@ SIGNATURES = {
     "regione_region_rows": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_int, c_int,
                                     _P, _P, c_int, _P, _P, c_int, _P, _P]),
     "regione_gather": (c_int, [_P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int64, _P, _P, _P]),
+    "regione_gather_multi": (c_int, [_P, _P, c_int, _P, _P, c_int, c_int64, c_int64, c_int64, c_int64, _P, _P]),
     "regione_scatter": (c_int, [_P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int64, _P, _P, _P]),
     "regione_rikv_store": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
     "regione_region_attention_workspace": (c_size_t, [c_int] * 6),
@@ -157,6 +158,23 @@ def gather(src, idx, n, dst, dev_status=None, stream=None):
         _ptr(src, None, "src"), _ptr(idx, torch.int32, "idx"), _ptr(n, torch.int32, "n"), B,
         src.shape[1], idx.shape[1], dst.shape[1], _row_bytes(src), _ptr(dst, src.dtype, "dst"),
         _ptr(dev_status, torch.int32), _stream(stream)), "regione_gather")
+
+
+def gather_multi(srcs, idx, n, dsts, dev_status=None, stream=None):
+    """dsts[i][b, j] = srcs[i][b, idx[b, j]] for up to 4 same-shaped tensors, one launch."""
+    torch = _torch()
+    k = len(srcs)
+    if k != len(dsts) or not 1 <= k <= 4:
+        raise RegionEError("gather_multi takes 1 to 4 (src, dst) pairs")
+    for s_, d_ in zip(srcs, dsts):
+        if s_.shape != srcs[0].shape or d_.shape != dsts[0].shape or s_.dtype != d_.dtype:
+            raise RegionEError("gather_multi: tensors must share shape and dtype")
+    sp = (c_void_p * k)(*[_ptr(t, None, "src").value for t in srcs])
+    dp = (c_void_p * k)(*[_ptr(t, None, "dst").value for t in dsts])
+    _check(load().regione_gather_multi(
+        sp, dp, k, _ptr(idx, torch.int32, "idx"), _ptr(n, torch.int32, "n"), srcs[0].shape[0],
+        srcs[0].shape[1], idx.shape[1], dsts[0].shape[1], _row_bytes(srcs[0]),
+        _ptr(dev_status, torch.int32), _stream(stream)), "regione_gather_multi")
 
 
 def scatter(src, idx, n, dst, dev_status=None, stream=None):

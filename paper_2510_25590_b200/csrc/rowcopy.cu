@@ -19,15 +19,20 @@ struct RowCopyPair {
     uint4* dst;
 };
 
+constexpr int kMaxPairs = 4;                 // tensors sharing one index list in one launch
+struct RowCopyPairs {
+    RowCopyPair p[kMaxPairs];
+};
+
 // GATHER: dst[b, j] = src[b, idx[b, j]];  !GATHER: dst[b, idx[b, j]] = src[b, j].
 // `idx_rows` bounds the indexed side, `cap` the dense side.  blockIdx.z picks the tensor pair.
 template <bool GATHER>
 __global__ void __launch_bounds__(kCopyThreads)
-row_copy_kernel(RowCopyPair p0, RowCopyPair p1, const int32_t* __restrict__ idx,
+row_copy_kernel(const RowCopyPairs pairs, const int32_t* __restrict__ idx,
                 const int32_t* __restrict__ n, long long idx_rows, long long idx_stride,
                 long long cap, int cpr, int32_t* dev_status) {
     const int b = blockIdx.y;
-    const RowCopyPair p = (blockIdx.z == 0) ? p0 : p1;
+    const RowCopyPair p = pairs.p[blockIdx.z];
     long long live = n[b];
     if (live < 0 || live > cap) {
         if (threadIdx.x == 0 && blockIdx.x == 0) record_status(dev_status, REGIONE_DEV_BOUNDS);
@@ -73,7 +78,7 @@ row_copy_kernel(RowCopyPair p0, RowCopyPair p1, const int32_t* __restrict__ idx,
 }
 
 template <bool GATHER>
-static int launch_row_copy(RowCopyPair p0, RowCopyPair p1, int pairs, const int32_t* idx,
+static int launch_row_copy(const RowCopyPairs& ps, int pairs, const int32_t* idx,
                            const int32_t* n, int B, long long idx_rows, long long idx_stride,
                            long long cap, long long row_bytes, int32_t* dev_status, void* stream) {
     const long long cpr = row_bytes / 16;
@@ -82,7 +87,7 @@ static int launch_row_copy(RowCopyPair p0, RowCopyPair p1, int pairs, const int3
     if (cap * cpr + per_block >= 0x7fffffffLL) return REGIONE_UNSUPPORTED;
     dim3 grid((unsigned)blocks, (unsigned)B, (unsigned)pairs);
     row_copy_kernel<GATHER><<<grid, kCopyThreads, 0, (cudaStream_t)stream>>>(
-        p0, p1, idx, n, idx_rows, idx_stride, cap, (int)cpr, dev_status);
+        ps, idx, n, idx_rows, idx_stride, cap, (int)cpr, dev_status);
     return launch_status(cudaGetLastError());
 }
 
@@ -106,8 +111,9 @@ extern "C" int regione_gather(const void* src, const int32_t* idx, const int32_t
     if (s != REGIONE_OK) return s;
     if (idx_stride < dst_rows_cap) return REGIONE_INVALID_ARG;
     if (B == 0 || dst_rows_cap == 0) return REGIONE_OK;
-    RowCopyPair p{(const uint4*)src, (uint4*)dst};
-    return launch_row_copy<true>(p, p, 1, idx, n, B, src_rows, idx_stride, dst_rows_cap, row_bytes,
+    RowCopyPairs ps = {};
+    ps.p[0] = RowCopyPair{(const uint4*)src, (uint4*)dst};
+    return launch_row_copy<true>(ps, 1, idx, n, B, src_rows, idx_stride, dst_rows_cap, row_bytes,
                                  dev_status, stream);
 }
 
@@ -118,8 +124,9 @@ extern "C" int regione_scatter(const void* src, const int32_t* idx, const int32_
     if (s != REGIONE_OK) return s;
     if (idx_stride < src_rows_cap) return REGIONE_INVALID_ARG;
     if (B == 0 || src_rows_cap == 0) return REGIONE_OK;
-    RowCopyPair p{(const uint4*)src, (uint4*)dst};
-    return launch_row_copy<false>(p, p, 1, idx, n, B, dst_rows, idx_stride, src_rows_cap, row_bytes,
+    RowCopyPairs ps = {};
+    ps.p[0] = RowCopyPair{(const uint4*)src, (uint4*)dst};
+    return launch_row_copy<false>(ps, 1, idx, n, B, dst_rows, idx_stride, src_rows_cap, row_bytes,
                                   dev_status, stream);
 }
 
@@ -135,8 +142,26 @@ extern "C" int regione_rikv_store(const regione_bf16* k_full, const regione_bf16
     const long long row_bytes = (long long)H * D * 2;
     if (row_bytes % 16 != 0 || B > 65535) return REGIONE_UNSUPPORTED;
     if (B == 0 || Nc_cap == 0) return REGIONE_OK;
-    RowCopyPair pk{(const uint4*)k_full, (uint4*)k_cache};
-    RowCopyPair pv{(const uint4*)v_full, (uint4*)v_cache};
-    return launch_row_copy<true>(pk, pv, 2, keep_rows, n_keep, B, N_full, Nc_cap, Nc_cap, row_bytes,
+    RowCopyPairs ps = {};
+    ps.p[0] = RowCopyPair{(const uint4*)k_full, (uint4*)k_cache};
+    ps.p[1] = RowCopyPair{(const uint4*)v_full, (uint4*)v_cache};
+    return launch_row_copy<true>(ps, 2, keep_rows, n_keep, B, N_full, Nc_cap, Nc_cap, row_bytes,
+                                 dev_status, stream);
+}
+
+extern "C" int regione_gather_multi(const void* const* srcs, void* const* dsts, int n_tensors,
+                                    const int32_t* idx, const int32_t* n, int B, int64_t src_rows,
+                                    int64_t idx_stride, int64_t dst_rows_cap, int64_t row_bytes,
+                                    int32_t* dev_status, void* stream) {
+    if (!srcs || !dsts || n_tensors < 1 || n_tensors > kMaxPairs) return REGIONE_INVALID_ARG;
+    RowCopyPairs ps = {};
+    for (int i = 0; i < n_tensors; ++i) {
+        int s = check_rows(srcs[i], idx, n, dsts[i], B, src_rows, idx_stride, dst_rows_cap, row_bytes);
+        if (s != REGIONE_OK) return s;
+        ps.p[i] = RowCopyPair{(const uint4*)srcs[i], (uint4*)dsts[i]};
+    }
+    if (idx_stride < dst_rows_cap) return REGIONE_INVALID_ARG;
+    if (B == 0 || dst_rows_cap == 0) return REGIONE_OK;
+    return launch_row_copy<true>(ps, n_tensors, idx, n, B, src_rows, idx_stride, dst_rows_cap, row_bytes,
                                  dev_status, stream);
 }

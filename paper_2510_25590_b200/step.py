@@ -4,8 +4,8 @@ This is call sequencing and buffer ownership only (torch tensors are device
 buffers): every operation runs in the library's kernels.  The sequence follows
 Algorithm 1 of the paper for one layer:
 
-  partition -> row lists -> gather X^E, v^E -> RIKV store -> gather Q/K/V of the
-  recomputed rows -> region attention -> scatter the attention rows back ->
+  partition -> row lists -> gather X^E, v^E (one launch) -> RIKV store -> gather Q/K/V of the
+  recomputed rows (one launch) -> region attention -> scatter the attention rows back ->
   velocity decay + Euler update -> merge with one-step-predicted unedited tokens.
 
 No step needs a host round trip: per-request counts stay in device memory.
@@ -93,13 +93,12 @@ class RegionStep:
         b.region_rows(self.edit_idx, self.keep_idx, self.n_edit, s.n_text, s.n_ref, s.membership,
                       self.query_rows, self.n_q, self.cache_rows, self.n_cache, dev_status=st,
                       stream=stream)
-        b.gather(x_t, self.edit_idx, self.n_edit, self.x_e, dev_status=st, stream=stream)
-        b.gather(v, self.edit_idx, self.n_edit, self.v_e, dev_status=st, stream=stream)
+        b.gather_multi([x_t, v], self.edit_idx, self.n_edit, [self.x_e, self.v_e], dev_status=st,
+                       stream=stream)
         b.rikv_store(k_full, v_full, self.cache_rows, self.n_cache, self.k_cache, self.v_cache,
                      dev_status=st, stream=stream)
-        b.gather(q_full, self.query_rows, self.n_q, self.q_e, dev_status=st, stream=stream)
-        b.gather(k_full, self.query_rows, self.n_q, self.k_fresh, dev_status=st, stream=stream)
-        b.gather(v_full, self.query_rows, self.n_q, self.v_fresh, dev_status=st, stream=stream)
+        b.gather_multi([q_full, k_full, v_full], self.query_rows, self.n_q,
+                       [self.q_e, self.k_fresh, self.v_fresh], dev_status=st, stream=stream)
         if self.attention_events is not None:
             self.attention_events[0].record(stream)
         b.region_attention(self.q_e, self.k_fresh, self.v_fresh, self.k_cache, self.v_cache, self.n_q,
@@ -111,5 +110,5 @@ class RegionStep:
         b.velocity_decay(self.v_e, scale, dt, self.x_e, self.n_edit, v_cache_out=self.v_avd,
                          dev_status=st, stream=stream)
         b.merge(x_t, v, self.x_e, self.slot, dt_unedited, self.x_out, dev_status=st, stream=stream)
-        self.launches += 12
+        self.launches += 10          # kernels launched (the attention call launches two)
         return self.x_out

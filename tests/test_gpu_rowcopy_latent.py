@@ -140,3 +140,24 @@ def test_gamma_fit(S, T1, n):
     want_n, want_g = orc.gamma_fit(v, dt)
     assert np.allclose(norms.cpu().numpy(), want_n, rtol=2e-6)
     assert np.allclose(gamma.cpu().numpy(), want_g, rtol=1e-5)
+
+
+def test_gather_multi_matches_single_gathers():
+    import torch
+    rng = np.random.default_rng(9)
+    B, rows, cap, inner = 2, 300, 120, (3, 64)
+    srcs = [dev_bf16(synth.bf16_round(rng.standard_normal((B, rows) + inner).astype(np.float32))) for _ in range(3)]
+    idx = torch.stack([torch.randperm(rows, device="cuda")[:cap].sort()[0] for _ in range(B)]).to(torch.int32).contiguous()
+    n = torch.tensor([cap, 77], dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    one = [torch.full((B, cap) + inner, -3.0, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    many = [t.clone() for t in one]
+    for s_, d_ in zip(srcs, one):
+        binding.gather(s_, idx, n, d_, dev_status=st)
+    binding.gather_multi(srcs, idx, n, many, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st[0]) == 0
+    for a, b_ in zip(one, many):
+        assert torch.equal(a, b_)
+    with pytest.raises(binding.RegionEError):
+        binding.gather_multi(srcs * 2, idx, n, many * 2)
