@@ -44,6 +44,7 @@
 // records REGIONE_DEV_TIMEOUT, all roles leave their loops, tensor memory is
 // released and the kernel ends normally.
 #include <cuda.h>
+#include <type_traits>
 
 #include <algorithm>
 
@@ -651,6 +652,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     const long long hi = pl.whole_items ? pl.total : min(pos + pl.chunk, pl.total);
     if (pos >= hi) return;                              // uniform for the CTA
 
+    ptx::grid_launch_dependents();                      // the merge kernel may queue up behind this CTA
     if (threadIdx.x == 0) ctrl->abort_flag = 0;
     if (warp == 9) {
         ptx::tmem_alloc(ptx::smem_addr(&ctrl->tmem_base), 512);
@@ -684,10 +686,17 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
 // Merges the workspace slots of the items that were spread over several shares:
 // out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  One warp per (request, query row, head); a
 // lane owns D / 32 consecutive columns.  `grid_main` is the grid of the attention kernel, from which
-// the same plan (share length, slots per item) is derived.
+// the same plan (share length, slots per item) is derived.  The kernel is launched behind the
+// attention kernel with programmatic serialization: the plan is computed from the launch's inputs
+// while that kernel may still run, the slots are read after the dependency wait; all slots'
+// loads are issued before the first use, so a warp pays one memory round trip, not one per slot.
+constexpr int kCombineMaxSlots = 8;      // upper bound of AttnParams::max_slots
+
 template <int D>
 __global__ void __launch_bounds__(256)
 region_attention_combine_kernel(const AttnParams p, int grid_main) {
+    constexpr int E = D / 32;
+    using Vec = typename std::conditional<E == 4, float4, float2>::type;
     const int b = blockIdx.z;
     const int lane = threadIdx.x & 31;
     const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);     // (row, head) pair
@@ -705,35 +714,50 @@ region_attention_combine_kernel(const AttnParams p, int grid_main) {
     const int len = pl.item_len(r);
     const long long first = base + ((long long)h * r.np + qp) * len;
     const int c_first = (int)(first / pl.chunk);
-    const int n_slots = (int)((first + len - 1) / pl.chunk) - c_first + 1;
+    const int n_slots = min((int)((first + len - 1) / pl.chunk) - c_first + 1, kCombineMaxSlots);
     if (n_slots == 1) return;                        // written directly by the attention kernel
     const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + qp;
     const size_t prow0 = item_idx * p.max_slots * (2 * kBM) + (qrow - qp * 2 * kBM);
-    constexpr int E = D / 32;
-    float M = -INFINITY;
-    for (int s = 0; s < n_slots; ++s) {
-        const float2 ml = p.part_ml[prow0 + (size_t)s * (2 * kBM)];
-        if (ml.y > 0.f) M = fmaxf(M, ml.x);
+
+    ptx::grid_dependency_wait();
+
+    float2 ml[kCombineMaxSlots];
+    Vec o[kCombineMaxSlots];
+#pragma unroll
+    for (int s = 0; s < kCombineMaxSlots; ++s) {
+        if (s < n_slots) {
+            const size_t prow = prow0 + (size_t)s * (2 * kBM);
+            ml[s] = p.part_ml[prow];
+            o[s] = *reinterpret_cast<const Vec*>(p.part_o + prow * D + lane * E);
+        }
     }
+    float M = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < kCombineMaxSlots; ++s)
+        if (s < n_slots && ml[s].y > 0.f) M = fmaxf(M, ml[s].x);
     float acc[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
     float L = 0.f;
-    for (int s = 0; s < n_slots; ++s) {
-        const size_t prow = prow0 + (size_t)s * (2 * kBM);
-        const float2 ml = p.part_ml[prow];
-        if (!(ml.y > 0.f)) continue;
-        const float wgt = fast_exp2(ml.x - M);
-        L = fmaf(wgt, ml.y, L);
-        const float* po = p.part_o + prow * D + lane * E;
 #pragma unroll
-        for (int e = 0; e < E; ++e) acc[e] = fmaf(wgt, po[e], acc[e]);
+    for (int s = 0; s < kCombineMaxSlots; ++s) {
+        if (s < n_slots && ml[s].y > 0.f) {           // a slot without keys carries no weight
+            const float wgt = fast_exp2(ml[s].x - M);
+            L = fmaf(wgt, ml[s].y, L);
+            const float* po = reinterpret_cast<const float*>(&o[s]);
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[e] = fmaf(wgt, po[e], acc[e]);
+        }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
     uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D + lane * E;
+    uint32_t packed[E / 2];
 #pragma unroll
-    for (int e = 0; e < E; e += 2)
-        *reinterpret_cast<uint32_t*>(orow + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
+    for (int e = 0; e < E; e += 2) packed[e / 2] = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
+    if constexpr (E == 4)
+        *reinterpret_cast<uint2*>(orow) = make_uint2(packed[0], packed[1]);
+    else
+        *reinterpret_cast<uint32_t*>(orow) = packed[0];
 }
 
 // ---- host side ---------------------------------------------------------------------------------
@@ -826,9 +850,21 @@ static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, c
     region_attention_tc_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, st>>>(
         maps[0], maps[1], maps[2], maps[3], maps[4], prm);
     if (cudaGetLastError() != cudaSuccess) return REGIONE_CUDA_ERROR;
+    // the merge kernel may become resident while the attention kernel drains (it waits for that
+    // kernel's completion before it reads a slot)
     const long long warps = (long long)prm.Nq_cap * prm.H;
-    dim3 cgrid((unsigned)((warps + 7) / 8), 1, prm.B);
-    region_attention_combine_kernel<D><<<cgrid, 256, 0, st>>>(prm, grid);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((warps + 7) / 8), 1, prm.B);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, region_attention_combine_kernel<D>, prm, grid) != cudaSuccess)
+        return REGIONE_CUDA_ERROR;
     return launch_status(cudaGetLastError());
 }
 
