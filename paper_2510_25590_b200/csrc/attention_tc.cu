@@ -541,63 +541,85 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t][1]));
             }
         }
-        // epilogue (rows past n_q are not written)
-        const int qrow = q0 + t * kBM + row;
-        const bool live = qrow < nq;
+        // epilogue (rows past n_q are not written).  A thread holds one row, so storing straight
+        // from registers would touch 32 different rows per warp instruction; instead each warp
+        // passes 128-byte row pieces through its own 4 KB corner of the (now idle) query tile in
+        // shared memory and stores four whole pieces per instruction.
+        const int wrow0 = q0 + t * kBM + ((warp & 3) << 5);         // first query row of this warp
+        const int live_rows = min(max(nq - wrow0, 0), 32);
+        const bool live = lane < live_rows;
         if (n_tiles > 0 && ok) {
             ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status);
             if (ok) ptx::tc_fence_after_sync();
         }
+        uint8_t* const stage = smem_gen + t * kTileBytes + (warp & 3) * (kTileBytes / 4);
+        auto store_pieces = [&](const uint4 (&v)[8], uint8_t* g_row0, size_t row_stride) {
+            // piece q of row r sits at 16-byte column q ^ (r & 7): both the row-wise writes and
+            // the piece-wise reads are free of bank conflicts without padding
+            uint4* dst = reinterpret_cast<uint4*>(stage + lane * 128);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) dst[q ^ (lane & 7)] = v[q];
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int rr = i * 4 + (lane >> 3);
+                const uint4 x = *reinterpret_cast<const uint4*>(stage + rr * 128 +
+                                                                 (((lane & 7) ^ (rr & 7)) << 4));
+                if (rr < live_rows)
+                    *reinterpret_cast<uint4*>(g_row0 + rr * row_stride + (lane & 7) * 16) = x;
+            }
+            __syncwarp();
+        };
         if (direct) {
             // O / l -> bf16 -> out
-            uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D;
+            const size_t row_stride = (size_t)p.H * D * 2;
+            uint8_t* g_row0 = reinterpret_cast<uint8_t*>(p.out) +
+                              (((size_t)b * p.Nq_cap + wrow0) * p.H + h) * D * 2;
             if (n_tiles == 0) {
                 if (live)
                     for (int q = 0; q < D / 8; ++q)
-                        reinterpret_cast<uint4*>(orow)[q] = make_uint4(0, 0, 0, 0);
+                        reinterpret_cast<uint4*>(g_row0 + lane * row_stride)[q] = make_uint4(0, 0, 0, 0);
             } else if (ok) {
                 const float inv = l > 0.f ? 1.f / l : 0.f;
-                uint32_t r[32];
-#pragma unroll
-                for (int ch = 0; ch < D / 32; ++ch) {
-                    ptx::tmem_ld32(tO + ch * 32, r);
+#pragma unroll 1
+                for (int c64 = 0; c64 < D / 64; ++c64) {
+                    uint32_t r[64];
+                    ptx::tmem_ld32(tO + c64 * 64, r);
+                    ptx::tmem_ld32(tO + c64 * 64 + 32, r + 32);
                     ptx::tmem_wait_ld();
-                    if (live) {
+                    uint4 v[8];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            uint4 o;
-                            o.x = pack_bf16x2(__uint_as_float(r[8 * q + 0]) * inv, __uint_as_float(r[8 * q + 1]) * inv);
-                            o.y = pack_bf16x2(__uint_as_float(r[8 * q + 2]) * inv, __uint_as_float(r[8 * q + 3]) * inv);
-                            o.z = pack_bf16x2(__uint_as_float(r[8 * q + 4]) * inv, __uint_as_float(r[8 * q + 5]) * inv);
-                            o.w = pack_bf16x2(__uint_as_float(r[8 * q + 6]) * inv, __uint_as_float(r[8 * q + 7]) * inv);
-                            reinterpret_cast<uint4*>(orow + ch * 32)[q] = o;
-                        }
+                    for (int q = 0; q < 8; ++q) {
+                        v[q].x = pack_bf16x2(__uint_as_float(r[8 * q + 0]) * inv, __uint_as_float(r[8 * q + 1]) * inv);
+                        v[q].y = pack_bf16x2(__uint_as_float(r[8 * q + 2]) * inv, __uint_as_float(r[8 * q + 3]) * inv);
+                        v[q].z = pack_bf16x2(__uint_as_float(r[8 * q + 4]) * inv, __uint_as_float(r[8 * q + 5]) * inv);
+                        v[q].w = pack_bf16x2(__uint_as_float(r[8 * q + 6]) * inv, __uint_as_float(r[8 * q + 7]) * inv);
                     }
+                    store_pieces(v, g_row0 + c64 * 128, row_stride);
                 }
             }
         } else {
             // unnormalised O and (m, l) of this segment -> its workspace slot
             const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + it.qp;
-            const size_t prow = (item_idx * p.max_slots + slot) * (2 * kBM) + t * kBM + row;
+            const size_t prow_w = (item_idx * p.max_slots + slot) * (2 * kBM) + t * kBM + ((warp & 3) << 5);
             if (n_tiles == 0) {
-                if (live) p.part_ml[prow] = make_float2(-INFINITY, 0.f);
+                if (live) p.part_ml[prow_w + lane] = make_float2(-INFINITY, 0.f);
             } else if (ok) {
-                float* po = p.part_o + prow * D;
-                uint32_t r[32];
-#pragma unroll
+                uint8_t* g_row0 = reinterpret_cast<uint8_t*>(p.part_o + prow_w * D);
+#pragma unroll 1
                 for (int ch = 0; ch < D / 32; ++ch) {
+                    uint32_t r[32];
                     ptx::tmem_ld32(tO + ch * 32, r);
                     ptx::tmem_wait_ld();
-                    if (live) {
+                    uint4 v[8];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            reinterpret_cast<uint4*>(po + ch * 32)[q] =
-                                make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-                    }
+                    for (int q = 0; q < 8; ++q) v[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                    store_pieces(v, g_row0 + ch * 128, (size_t)D * 4);
                 }
-                if (live) p.part_ml[prow] = make_float2(m, l);
+                if (live) p.part_ml[prow_w + lane] = make_float2(m, l);
             }
         }
+        ptx::fence_proxy_async_smem();      // the next segment's query tile arrives by TMA
     }
 
     // ---- end of the segment: every role is done with shared and tensor memory ----
