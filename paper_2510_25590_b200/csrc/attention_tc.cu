@@ -32,10 +32,12 @@
 //
 // Scheduling: the kernel is persistent, one CTA per SM.  A "step" is one key tile of one
 // (request, head, query pair) item; all steps of the launch form one sequence, item after item,
-// which is cut into equal contiguous shares, one per CTA (a stream-K decomposition: the grid is
-// always one balanced wave, whatever the number of items).  A CTA's share is a few segments,
-// each a run of key tiles of one item.  A segment that covers its item completely writes the
-// output rows directly; otherwise it writes its unnormalised output and (max, sum) pair to a
+// laid out on a cost axis (a step of a pair with one live query tile costs a little less than a
+// step of a full pair, and every item starts with a fixed cost for draining and refilling the
+// pipeline), which is cut into equal contiguous shares, one per CTA (a stream-K decomposition:
+// the grid is always one balanced wave, whatever the number of items).  A CTA's share is a few
+// segments, each a run of key tiles of one item.  A segment that covers its item completely writes
+// the output rows directly; otherwise it writes its unnormalised output and (max, sum) pair to a
 // slot of the caller's workspace and a small second kernel merges the slots of such items.  The
 // share length is bounded below so that no item is spread over more slots than the workspace
 // holds.  Counts live in device memory, so every CTA derives the same plan from them.
@@ -82,6 +84,12 @@ struct AttnCtrl {
     int abort_flag;
 };
 
+// What share c tells the merge kernel: the item that the boundary between shares c - 1 and c
+// cuts, if c is the second share of that item (so every cut item is named exactly once).
+struct alignas(16) CutItem {
+    int valid, b, h, qp, n_slots, nq, pad0, pad1;
+};
+
 struct AttnParams {
     const int32_t* n_q;
     const int32_t* n_fresh;
@@ -94,14 +102,26 @@ struct AttnParams {
     int32_t* dev_status;
     float* part_o;       // [B, H, P_cap, max_slots, 256, D] unnormalised outputs
     float2* part_ml;     // [B, H, P_cap, max_slots, 256]    (running max in the exp2 domain, sum)
+    CutItem* cut;        // [grid] the item that the start of each share cuts, for the merge kernel
 };
 
+
 // ---- the plan every CTA (and the merge kernel) derives from the device-side counts ------------
+// Shares are cut on a cost axis measured in ticks, not in steps, so that they take about the same
+// time: a key tile of a full query pair costs kTickPair, a key tile of a pair with one live query
+// tile kTickSingle (it is bound by the tile's dependency chain, not by the work), and every item
+// starts with kTickStart ticks that stand for the drain of the previous segment and the fill of the
+// new one (measured on the kernel: 2.3 us, 2.0 us and about 8 us).
+constexpr int kTickPair = 8, kTickSingle = 7, kTickStart = 28;
+
 struct ReqShape {
     int nq, nf, nc;      // clamped counts
     int np;              // live query pairs
     int nt_c, nt;        // cached key tiles, all key tiles
     long long items;     // H * np
+    int steps;           // steps of an item: max(nt, 1) (an item without keys writes zeros in one step)
+    int w_last;          // ticks per step of the last query pair
+    long long ticks_full, ticks_last, head_ticks, ticks;   // per full-pair item, last item, head, request
 };
 
 __device__ __forceinline__ ReqShape req_shape(const AttnParams& p, int b, bool* bad = nullptr) {
@@ -118,32 +138,34 @@ __device__ __forceinline__ ReqShape req_shape(const AttnParams& p, int b, bool* 
     r.nt_c = (nc + kBN - 1) / kBN;
     r.nt = r.nt_c + (nf + kBN - 1) / kBN;
     r.items = (long long)p.H * r.np;
+    r.steps = max(r.nt, 1);
+    r.w_last = (nq - (r.np - 1) * 2 * kBM > kBM) ? kTickPair : kTickSingle;
+    r.ticks_full = kTickStart + (long long)kTickPair * r.steps;
+    r.ticks_last = kTickStart + (long long)r.w_last * r.steps;
+    r.head_ticks = r.np > 0 ? (r.np - 1) * r.ticks_full + r.ticks_last : 0;
+    r.ticks = p.H * r.head_ticks;
     return r;
 }
 
-// How the launch's work is cut into one contiguous share per CTA.
-//  - whole items: when handing out whole items wastes at most 6 % of the grid's last round, each
-//    item counts as one step and is never split (no workspace traffic, no merge).
-//  - otherwise a step is one key tile of an item (an item without keys still takes one step: it
-//    writes zeros) and shares may cut items; the share length is then at least
-//    ceil(longest item / (max_slots - 1)) so that an item never spans more than max_slots shares.
+// How the launch's work is cut into shares, one per CTA.
+//  - whole items: when handing out whole items wastes at most 6 % of the grid's last round, items
+//    are dealt round-robin and never split (no workspace traffic, no merge): positions count items.
+//  - otherwise positions count ticks and CTA c owns the steps whose first tick lies in
+//    [c * chunk, (c + 1) * chunk); shares may cut items.  The share length is bounded below so
+//    that an item never meets more than max_slots shares.
 struct Plan {
     bool whole_items;
     long long total, chunk;
-    __device__ __forceinline__ int item_len(const ReqShape& r) const {
-        return whole_items ? 1 : max(r.nt, 1);
-    }
 };
 
 __device__ __forceinline__ Plan plan_shares(const AttnParams& p, int grid, bool* bad = nullptr) {
     Plan pl;
-    long long items = 0, steps = 0;
-    int nt_max = 1;
+    long long items = 0, ticks = 0, span = 0;      // span: first tick of an item's last step, at most
     for (int b = 0; b < p.B; ++b) {
         const ReqShape r = req_shape(p, b, bad);
         items += r.items;
-        steps += r.items * max(r.nt, 1);
-        if (r.np > 0) nt_max = max(nt_max, r.nt);
+        ticks += r.ticks;
+        if (r.np > 0) span = max(span, (long long)(r.np > 1 ? kTickPair : r.w_last) * (r.steps - 1));
     }
     const long long per = (items + grid - 1) / grid;
     pl.whole_items = per * grid * 100 <= items * 106;
@@ -151,43 +173,94 @@ __device__ __forceinline__ Plan plan_shares(const AttnParams& p, int grid, bool*
         pl.total = items;
         pl.chunk = max(per, 1LL);
     } else {
-        pl.total = steps;
-        pl.chunk = (steps + grid - 1) / grid;
-        const long long floor_len = (nt_max + p.max_slots - 2) / (p.max_slots - 1);
+        pl.total = ticks;
+        pl.chunk = (ticks + grid - 1) / grid;
+        // an item meets at most span / chunk + 2 shares: keep that within max_slots; and a share is
+        // at least one step long, so that every share between an item's first and last holds a
+        // step of it (and writes its slot)
+        const long long floor_len = max(span / (p.max_slots - 1) + 1, (long long)kTickPair);
         if (pl.chunk < floor_len) pl.chunk = floor_len;
-        if (pl.chunk < 1) pl.chunk = 1;
     }
     return pl;
 }
 
-// The item that step `pos` belongs to.
-struct ItemAt {
+// The part of one item that a CTA works on.
+struct Segment {
     int b, h, qp;
-    int j0;              // position of `pos` inside the item
-    int len;             // steps of the item
-    long long first;     // first step of the item in the sequence
     ReqShape r;
+    int j_first, n_steps;   // steps [j_first, j_first + n_steps) of the item; n_steps may be 0
+    int slot, n_slots;      // this share's slot among the shares that hold steps of the item
+    long long next;         // position behind the item
 };
 
-__device__ __forceinline__ ItemAt item_at(const AttnParams& p, const Plan& pl, long long pos) {
-    ItemAt it;
+// Shares that hold steps of the item whose step 0 starts at tick `first_tick`.
+__device__ __forceinline__ void item_slots(const Plan& pl, long long first_tick, int w, int steps,
+                                           int& c_first, int& n_slots) {
+    c_first = (int)(first_tick / pl.chunk);
+    n_slots = (int)((first_tick + (long long)w * (steps - 1)) / pl.chunk) - c_first + 1;
+}
+
+// Whole-item plan: the item with index `idx`.
+__device__ __forceinline__ Segment segment_whole(const AttnParams& p, long long idx) {
+    Segment sg;
     long long base = 0;
     int b = 0;
     ReqShape r = req_shape(p, 0);
-    while (pos >= base + r.items * pl.item_len(r) && b + 1 < p.B) {
-        base += r.items * pl.item_len(r);
+    while (idx >= base + r.items && b + 1 < p.B) {
+        base += r.items;
         ++b;
         r = req_shape(p, b);
     }
-    it.b = b; it.r = r;
-    it.len = pl.item_len(r);
+    const long long item = idx - base;
+    sg.b = b; sg.r = r;
+    sg.h = r.np > 0 ? (int)(item / r.np) : 0;
+    sg.qp = (int)(item - (long long)sg.h * r.np);
+    sg.j_first = 0;
+    sg.n_steps = r.np > 0 ? r.steps : 0;
+    sg.slot = 0; sg.n_slots = 1;
+    sg.next = idx + 1;
+    return sg;
+}
+
+// Tick plan: the item that contains tick `pos`, and the steps of it that share `c` owns.
+__device__ __forceinline__ Segment segment_ticks(const AttnParams& p, const Plan& pl, long long pos,
+                                                 int c) {
+    Segment sg;
+    long long base = 0;
+    int b = 0;
+    ReqShape r = req_shape(p, 0);
+    while (pos >= base + r.ticks && b + 1 < p.B) {
+        base += r.ticks;
+        ++b;
+        r = req_shape(p, b);
+    }
+    sg.b = b; sg.r = r;
+    if (r.np == 0) {                                  // nothing left behind the last live request
+        sg.h = sg.qp = sg.j_first = sg.n_steps = sg.slot = 0;
+        sg.n_slots = 1;
+        sg.next = pl.total;
+        return sg;
+    }
     const long long rel = pos - base;
-    const long long item = rel / it.len;
-    it.j0 = (int)(rel - item * it.len);
-    it.h = (int)(item / r.np);
-    it.qp = (int)(item - (long long)it.h * r.np);
-    it.first = base + item * it.len;
-    return it;
+    sg.h = (int)(rel / r.head_ticks);
+    const long long rem = rel - (long long)sg.h * r.head_ticks;
+    sg.qp = (int)min(rem / r.ticks_full, (long long)(r.np - 1));
+    const long long t0 = base + (long long)sg.h * r.head_ticks + (long long)sg.qp * r.ticks_full;
+    const bool last = sg.qp == r.np - 1;
+    const int w = last ? r.w_last : kTickPair;
+    const long long first_tick = t0 + kTickStart;
+    const long long lo = (long long)c * pl.chunk, hi = lo + pl.chunk;
+    long long s_lo = lo <= first_tick ? 0 : (lo - first_tick + w - 1) / w;
+    long long s_hi = hi <= first_tick ? 0 : (hi - first_tick + w - 1) / w;
+    s_lo = min(s_lo, (long long)r.steps);
+    s_hi = min(s_hi, (long long)r.steps);
+    sg.j_first = (int)s_lo;
+    sg.n_steps = (int)(s_hi - s_lo);
+    int c_first;
+    item_slots(pl, first_tick, w, r.steps, c_first, sg.n_slots);
+    sg.slot = c - c_first;
+    sg.next = t0 + (last ? r.ticks_last : r.ticks_full);
+    return sg;
 }
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
@@ -273,21 +346,32 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     const CUtensorMap& tm_vf = *tm_vf_;
     const CUtensorMap& tm_kc = *tm_kc_;
     const CUtensorMap& tm_vc = *tm_vc_;
+    bool first_segment = true;
     while (pos < hi) {
     // ---- the segment: key tiles [j_first, j_first + n_tiles) of item (b, h, query pair) ----
-    const ItemAt it = item_at(p, pl, pos);
-    const int seg_len = (int)min((long long)(it.len - it.j0), hi - pos);
+    const Segment it = pl.whole_items ? segment_whole(p, pos) : segment_ticks(p, pl, pos, (int)blockIdx.x);
+    if (first_segment && SOFTMAX_WG && threadIdx.x == 0) {
+        // tell the merge kernel which item the start of this share cuts
+        CutItem ci;
+        ci.valid = (!pl.whole_items && it.r.np > 0 && it.n_slots >= 2 && it.slot == 1) ? 1 : 0;
+        ci.b = it.b; ci.h = it.h; ci.qp = it.qp; ci.n_slots = it.n_slots; ci.nq = it.r.nq;
+        ci.pad0 = ci.pad1 = 0;
+        p.cut[blockIdx.x] = ci;
+    }
+    first_segment = false;
+    if (it.n_steps == 0) {                              // (uniform for the CTA)
+        pos = pl.whole_items ? pos + gridDim.x : it.next;
+        continue;
+    }
     const int b = it.b, h = it.h;
     const int q0 = it.qp * (2 * kBM);
     const int nq = it.r.nq, nf = it.r.nf, nc = it.r.nc, nt_c = it.r.nt_c;
     const int ntq = (nq - q0 > kBM) ? 2 : 1;            // live query tiles of this segment
-    const int j_first = it.j0;
-    const int n_tiles = pl.whole_items ? it.r.nt : (it.r.nt == 0 ? 0 : seg_len);
+    const int j_first = it.j_first;
+    const int n_tiles = it.r.nt == 0 ? 0 : it.n_steps;
     // slot of this segment among the shares that touch the item; a lone segment writes the output
-    const int c_first = (int)(it.first / pl.chunk);
-    const int n_slots = pl.whole_items ? 1 : (int)((it.first + it.len - 1) / pl.chunk) - c_first + 1;
-    const int slot = (int)blockIdx.x - c_first;
-    const bool direct = n_slots == 1;
+    const int slot = it.slot;
+    const bool direct = it.n_slots == 1;
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(ptx::smem_addr(&ctrl->q_full), 1);
@@ -640,7 +724,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             ptx::mbar_inval(ptx::smem_addr(&ctrl->turn[t]));
         }
     }
-    pos += pl.whole_items ? (long long)gridDim.x : (long long)seg_len;
+    pos = pl.whole_items ? pos + gridDim.x : it.next;
     if (*abort_flag) break;
     }   // segments
 }
@@ -664,7 +748,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     volatile int* abort_flag = &ctrl->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // this CTA's share [pos, hi) of the step sequence
+    // this CTA's share [pos, hi) of the item sequence or of the cost axis
     bool bad = false;
     const Plan pl = plan_shares(p, gridDim.x, &bad);
     if (bad && blockIdx.x == 0 && threadIdx.x == 0) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
@@ -672,7 +756,10 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     // neighbouring items, which share K/V tiles in L2; a share of steps is one contiguous range)
     long long pos = pl.whole_items ? (long long)blockIdx.x : (long long)blockIdx.x * pl.chunk;
     const long long hi = pl.whole_items ? pl.total : min(pos + pl.chunk, pl.total);
-    if (pos >= hi) return;                              // uniform for the CTA
+    if (pos >= hi) {                                    // uniform for the CTA
+        if (threadIdx.x == 0) p.cut[blockIdx.x].valid = 0;
+        return;
+    }
 
     ptx::grid_launch_dependents();                      // the merge kernel may queue up behind this CTA
     if (threadIdx.x == 0) ctrl->abort_flag = 0;
@@ -706,42 +793,34 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
 }
 
 // Merges the workspace slots of the items that were spread over several shares:
-// out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  One warp per (request, query row, head); a
-// lane owns D / 32 consecutive columns.  `grid_main` is the grid of the attention kernel, from which
-// the same plan (share length, slots per item) is derived.  The kernel is launched behind the
-// attention kernel with programmatic serialization: the plan is computed from the launch's inputs
-// while that kernel may still run, the slots are read after the dependency wait; all slots'
-// loads are issued before the first use, so a warp pays one memory round trip, not one per slot.
+// out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  blockIdx.x + 1 names a share boundary; the
+// attention kernel has left the item cut there (if any) in `cut`.  One warp per query row of the
+// item's pair of tiles (blockIdx.y * 8 + warp); a lane owns D / 32 consecutive columns.  The kernel
+// is launched behind the attention kernel with programmatic serialization and reads nothing before
+// the dependency wait; all slots' loads are issued before the first use, so a warp pays one
+// memory round trip, not one per slot.
 constexpr int kCombineMaxSlots = 8;      // upper bound of AttnParams::max_slots
 
 template <int D>
 __global__ void __launch_bounds__(256)
-region_attention_combine_kernel(const AttnParams p, int grid_main) {
+region_attention_combine_kernel(const AttnParams p) {
     constexpr int E = D / 32;
     using Vec = typename std::conditional<E == 4, float4, float2>::type;
-    const int b = blockIdx.z;
-    const int lane = threadIdx.x & 31;
-    const long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);     // (row, head) pair
-    const int qrow = (int)(w / p.H), h = (int)(w % p.H);
-    const ReqShape r = req_shape(p, b);
-    if (qrow >= r.nq) return;
-    const Plan pl = plan_shares(p, grid_main);
-    if (pl.whole_items) return;                      // nothing was split
-    long long base = 0;
-    for (int bb = 0; bb < b; ++bb) {
-        const ReqShape rb = req_shape(p, bb);
-        base += rb.items * pl.item_len(rb);
-    }
-    const int qp = qrow / (2 * kBM);
-    const int len = pl.item_len(r);
-    const long long first = base + ((long long)h * r.np + qp) * len;
-    const int c_first = (int)(first / pl.chunk);
-    const int n_slots = min((int)((first + len - 1) / pl.chunk) - c_first + 1, kCombineMaxSlots);
-    if (n_slots == 1) return;                        // written directly by the attention kernel
-    const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + qp;
-    const size_t prow0 = item_idx * p.max_slots * (2 * kBM) + (qrow - qp * 2 * kBM);
-
     ptx::grid_dependency_wait();
+    const int4* cp = reinterpret_cast<const int4*>(p.cut + blockIdx.x + 1);
+    const int4 c0 = cp[0], c1 = cp[1];
+    const int b = c0.y, h = c0.z, qp = c0.w, n_slots = c1.x, nq = c1.y;
+    // (the fields are checked so that a table left incomplete by an aborted launch cannot send
+    // this kernel out of bounds)
+    if (c0.x != 1 || b < 0 || b >= p.B || h < 0 || h >= p.H || qp < 0 || qp >= p.P_cap ||
+        n_slots < 2 || n_slots > p.max_slots || n_slots > kCombineMaxSlots || nq > p.Nq_cap)
+        return;
+    const int lane = threadIdx.x & 31;
+    const int r_local = blockIdx.y * 8 + (threadIdx.x >> 5);
+    const int qrow = qp * (2 * kBM) + r_local;
+    if (qrow >= nq) return;
+    const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + qp;
+    const size_t prow0 = item_idx * p.max_slots * (2 * kBM) + r_local;
 
     float2 ml[kCombineMaxSlots];
     Vec o[kCombineMaxSlots];
@@ -855,7 +934,8 @@ static inline size_t slot_rows(const LaunchPlan& lp, int B, int H) {
 size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D) {
     const LaunchPlan lp = plan_launch(B, Nq_cap, Nf_cap, Nc_cap, H);
     const size_t rows = slot_rows(lp, B, H);
-    return ((rows * D * sizeof(float) + 255) & ~(size_t)255) + rows * sizeof(float2);
+    return ((rows * D * sizeof(float) + 255) & ~(size_t)255) +
+           ((rows * sizeof(float2) + 255) & ~(size_t)255) + (size_t)lp.grid * sizeof(CutItem);
 }
 
 template <int D>
@@ -874,9 +954,9 @@ static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, c
     if (cudaGetLastError() != cudaSuccess) return REGIONE_CUDA_ERROR;
     // the merge kernel may become resident while the attention kernel drains (it waits for that
     // kernel's completion before it reads a slot)
-    const long long warps = (long long)prm.Nq_cap * prm.H;
+    if (grid < 2) return launch_status(cudaGetLastError());     // a single share cuts nothing
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((warps + 7) / 8), 1, prm.B);
+    cfg.gridDim = dim3((unsigned)(grid - 1), (2 * kBM) / 8, 1);
     cfg.blockDim = dim3(256, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
@@ -885,7 +965,7 @@ static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, region_attention_combine_kernel<D>, prm, grid) != cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, region_attention_combine_kernel<D>, prm) != cudaSuccess)
         return REGIONE_CUDA_ERROR;
     return launch_status(cudaGetLastError());
 }
@@ -916,8 +996,10 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
     prm.out = out; prm.dev_status = dev_status;
     const size_t rows = slot_rows(lp, B, H);
     prm.part_o = reinterpret_cast<float*>(workspace);
-    prm.part_ml = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(workspace) +
-                                            ((rows * D * sizeof(float) + 255) & ~(size_t)255));
+    uint8_t* const ws = reinterpret_cast<uint8_t*>(workspace);
+    const size_t off_ml = (rows * D * sizeof(float) + 255) & ~(size_t)255;
+    prm.part_ml = reinterpret_cast<float2*>(ws + off_ml);
+    prm.cut = reinterpret_cast<CutItem*>(ws + off_ml + ((rows * sizeof(float2) + 255) & ~(size_t)255));
     return D == 64 ? launch_tc<64>(maps, prm, lp.grid, st) : launch_tc<128>(maps, prm, lp.grid, st);
 }
 
