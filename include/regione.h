@@ -183,11 +183,14 @@ int regione_rikv_store(const regione_bf16* k_full, const regione_bf16* v_full,
  * workspace       : dev, 256-byte aligned, at least
  *                   regione_region_attention_workspace(...) bytes.  It holds the
  *                   partial results of (request, head, query-tile pair) items whose
- *                   key range was shared between thread blocks; its contents need
- *                   not be initialised and mean nothing after the call.
+ *                   key range was shared between thread blocks, and a small table
+ *                   naming those items; its contents need not be initialised and
+ *                   mean nothing after the call.
  * D must be 64 or 128.  bf16 inputs, fp32 accumulation, probabilities rounded
  * to bf16 before the second product.  With no key at all a row is zero.
- * The call enqueues two kernels (attention, then the merge of shared items).
+ * The call enqueues two kernels (attention, then the merge of shared items; the
+ * second is launched with programmatic stream serialization, i.e. it may become
+ * resident while the first drains and waits for its completion on the device).
  */
 size_t regione_region_attention_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D);
 int regione_region_attention(const regione_bf16* q,
