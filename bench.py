@@ -224,21 +224,45 @@ def hbm_sweep(torch, binding, step, d, flush_l2, peak_gbs, iters=10):
           lambda: binding.gather(d["k"], idx, n_rows, dst))
     B, N, C = 32, 65536, 16
     g = torch.Generator(device="cuda"); g.manual_seed(7)
-    x_t, v, ref = ((torch.randn((B, N, C), device="cuda", generator=g)).to(bf) for _ in range(3))
+    ref = torch.randn((B, N, C), device="cuda", generator=g).to(bf)
+    # edit regions are spatially coherent, as in the paper's workloads: one ellipse per request on the
+    # 256 x 256 token grid covering 20 % of it, centre shifted from request to request; edited tokens get
+    # an estimate opposite to the reference (cosine -1), the others the reference itself (cosine +1)
+    side = 256
+    yy, xx = torch.meshgrid(torch.arange(side, device="cuda"), torch.arange(side, device="cuda"), indexing="ij")
+    ax, ay = 0.36 * side, 0.2 * side / (3.14159265 * 0.36)
+    blobs = []
+    for b in range(B):
+        cx, cy = side * (0.4 + 0.2 * ((b * 7) % 10) / 10), side * (0.4 + 0.2 * ((b * 3) % 10) / 10)
+        blobs.append((((xx - cx) / ax) ** 2 + ((yy - cy) / ay) ** 2 < 1.0).reshape(N))
+    blob = torch.stack(blobs)
+    x_t = torch.where(blob[:, :, None], -ref, ref)
+    v = torch.zeros_like(ref)
     mask = torch.empty((B, N), dtype=torch.uint8, device="cuda")
     e, k, sl = (torch.empty((B, N), dtype=i32, device="cuda") for _ in range(3))
     ne = torch.empty(B, dtype=i32, device="cuda")
     timed("partition, 2^21 tokens", B * N * (3 * C * 2 + 9),
           lambda: binding.partition(x_t, v, ref, 0.7, binding.METRIC_COSINE, 0.1, mask, e, k, sl, ne))
     n_e = int(ne.sum().item())
+    assert n_e == int(blob.sum().item()), (n_e, int(blob.sum().item()))
     x_e = torch.zeros((B, N, C), dtype=bf, device="cuda"); v_e = torch.zeros_like(x_e); v_c = torch.zeros_like(x_e)
-    timed("velocity_decay with cache refresh", n_e * 4 * C * 2,
-          lambda: binding.velocity_decay(v_e, 1.0, 1.0 / 28, x_e, ne, v_cache_out=v_c))
-    timed("velocity_decay reusing the cache", n_e * 3 * C * 2,
-          lambda: binding.velocity_decay(v_e, 0.9, 1.0 / 28, x_e, ne))
+    n_all = torch.full((B,), N, dtype=i32, device="cuda")          # every row live: traffic well above L2
+    timed("velocity_decay with cache refresh", B * N * 4 * C * 2,
+          lambda: binding.velocity_decay(v_e, 1.0, 1.0 / 28, x_e, n_all, v_cache_out=v_c))
+    timed("velocity_decay reusing the cache", B * N * 3 * C * 2,
+          lambda: binding.velocity_decay(v_e, 0.9, 1.0 / 28, x_e, n_all))
     x_out = torch.empty_like(x_t)
-    timed("merge", (B * N - n_e) * (3 * C * 2 + 4) + n_e * (2 * C * 2 + 4),
+    timed(f"merge, 2^21 tokens, elliptic regions ({100.0 * n_e / (B * N):.0f} % edited)",
+          (B * N - n_e) * (3 * C * 2 + 4) + n_e * (2 * C * 2 + 4),
           lambda: binding.merge(x_t, v, x_e, sl, 5.0 / 28, x_out))
+    # worst case for the merge: every token edited or not independently of its neighbours (random
+    # latents against the threshold), so the reads of the unedited rows skip single 32-byte rows
+    x_r, v_r = (torch.randn((B, N, C), device="cuda", generator=g).to(bf) for _ in range(2))
+    binding.partition(x_r, v_r, ref, 0.7, binding.METRIC_COSINE, 0.1, mask, e, k, sl, ne)
+    n_r = int(ne.sum().item())
+    timed(f"merge, 2^21 tokens, per-token random mask ({100.0 * n_r / (B * N):.0f} % edited)",
+          (B * N - n_r) * (3 * C * 2 + 4) + n_r * (2 * C * 2 + 4),
+          lambda: binding.merge(x_r, v_r, x_e, sl, 5.0 / 28, x_out))
     return out
 
 

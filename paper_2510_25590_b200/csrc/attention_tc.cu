@@ -748,6 +748,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     volatile int* abort_flag = &ctrl->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    grid_dependency_wait();                             // (everything below reads the launch's inputs)
     // this CTA's share [pos, hi) of the item sequence or of the cost axis
     bool bad = false;
     const Plan pl = plan_shares(p, gridDim.x, &bad);
@@ -761,7 +762,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         return;
     }
 
-    ptx::grid_launch_dependents();                      // the merge kernel may queue up behind this CTA
+    grid_launch_dependents();                      // the merge kernel may queue up behind this CTA
     if (threadIdx.x == 0) ctrl->abort_flag = 0;
     if (warp == 9) {
         ptx::tmem_alloc(ptx::smem_addr(&ctrl->tmem_base), 512);
@@ -806,7 +807,7 @@ __global__ void __launch_bounds__(256)
 region_attention_combine_kernel(const AttnParams p) {
     constexpr int E = D / 32;
     using Vec = typename std::conditional<E == 4, float4, float2>::type;
-    ptx::grid_dependency_wait();
+    grid_dependency_wait();
     const int4* cp = reinterpret_cast<const int4*>(p.cut + blockIdx.x + 1);
     const int4 c0 = cp[0], c1 = cp[1];
     const int b = c0.y, h = c0.z, qp = c0.w, n_slots = c1.x, nq = c1.y;
@@ -949,23 +950,16 @@ static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, c
             return REGIONE_CUDA_ERROR;
         configured = true;
     }
-    region_attention_tc_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, st>>>(
-        maps[0], maps[1], maps[2], maps[3], maps[4], prm);
-    if (cudaGetLastError() != cudaSuccess) return REGIONE_CUDA_ERROR;
+    if (launch_overlapped(region_attention_tc_kernel<D>, dim3(grid), dim3(kAttnThreads),
+                          Cfg::kSmemBytes, st, maps[0], maps[1], maps[2], maps[3], maps[4],
+                          prm) != cudaSuccess)
+        return REGIONE_CUDA_ERROR;
     // the merge kernel may become resident while the attention kernel drains (it waits for that
     // kernel's completion before it reads a slot)
     if (grid < 2) return launch_status(cudaGetLastError());     // a single share cuts nothing
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(grid - 1), (2 * kBM) / 8, 1);
-    cfg.blockDim = dim3(256, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, region_attention_combine_kernel<D>, prm) != cudaSuccess)
+    if (launch_overlapped(region_attention_combine_kernel<D>,
+                          dim3((unsigned)(grid - 1), (2 * kBM) / 8, 1), dim3(256), 0, st,
+                          prm) != cudaSuccess)
         return REGIONE_CUDA_ERROR;
     return launch_status(cudaGetLastError());
 }

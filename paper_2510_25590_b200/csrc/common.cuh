@@ -43,6 +43,35 @@ __device__ __forceinline__ uint4 ld_stream128(const void* p) {
     return r;
 }
 
+// Programmatic dependent launch.  Every kernel of the library starts with grid_dependency_wait():
+// it returns once the kernel ahead of it in the stream has completed and its writes are visible,
+// which is the ordinary stream order, but lets the launch itself (scheduling the grid, making its
+// thread blocks resident) overlap the tail of that kernel.  grid_launch_dependents() tells the
+// runtime that the kernel behind this one may be made resident.
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Launches `kernel` with programmatic stream serialization (see grid_dependency_wait).
+template <typename... Params, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline int launch_status(cudaError_t e) { return e == cudaSuccess ? REGIONE_OK : REGIONE_CUDA_ERROR; }

@@ -25,6 +25,8 @@ __global__ void __launch_bounds__(kLatThreads)
 velocity_decay_kernel(const uint4* __restrict__ v_in, float neg_dt_scale, uint4* __restrict__ x_e,
                       uint4* __restrict__ v_cache_out, const int32_t* __restrict__ n_edit,
                       int Ne_cap, int cpr, int32_t* dev_status) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int b = blockIdx.y;
     int ne = n_edit[b];
     if (ne < 0 || ne > Ne_cap) {
@@ -50,6 +52,8 @@ __global__ void __launch_bounds__(kLatThreads)
 merge_kernel(const uint4* x_full, const uint4* __restrict__ v_last,
              const uint4* __restrict__ x_e, const int32_t* __restrict__ slot, float neg_dt, int N,
              int Ne_cap, int cpr, uint4* x_out, int32_t* dev_status) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int b = blockIdx.y;
     const unsigned total = (unsigned)N * (unsigned)cpr;
     const unsigned base = blockIdx.x * (unsigned)(kLatThreads * kMergeUnroll) + threadIdx.x;
@@ -107,10 +111,9 @@ extern "C" int regione_velocity_decay(const regione_bf16* v_in, float scale, flo
     if (B == 0 || Ne_cap == 0) return REGIONE_OK;
     dim3 grid((unsigned)((total + kLatThreads - 1) / kLatThreads), B);
     // scale * v is formed first in fp32, then the Euler step: x - dt * (scale * v)
-    velocity_decay_kernel<<<grid, kLatThreads, 0, (cudaStream_t)stream>>>(
-        (const uint4*)v_in, -(dt * scale), (uint4*)x_e, (uint4*)v_cache_out, n_edit, Ne_cap,
-        (int)cpr, dev_status);
-    return launch_status(cudaGetLastError());
+    return launch_status(launch_overlapped(
+        velocity_decay_kernel, grid, dim3(kLatThreads), 0, (cudaStream_t)stream, (const uint4*)v_in,
+        -(dt * scale), (uint4*)x_e, (uint4*)v_cache_out, n_edit, Ne_cap, (int)cpr, dev_status));
 }
 
 extern "C" int regione_merge(const regione_bf16* x_full, const regione_bf16* v_last_full,
@@ -128,8 +131,8 @@ extern "C" int regione_merge(const regione_bf16* x_full, const regione_bf16* v_l
     if (B == 0) return REGIONE_OK;
     const long long per_block = (long long)kLatThreads * kMergeUnroll;
     dim3 grid((unsigned)((total + per_block - 1) / per_block), B);
-    merge_kernel<<<grid, kLatThreads, 0, (cudaStream_t)stream>>>(
-        (const uint4*)x_full, (const uint4*)v_last_full, (const uint4*)x_e, slot, -dt_unedited, N,
-        Ne_cap, (int)cpr, (uint4*)x_out, dev_status);
-    return launch_status(cudaGetLastError());
+    return launch_status(launch_overlapped(
+        merge_kernel, grid, dim3(kLatThreads), 0, (cudaStream_t)stream, (const uint4*)x_full,
+        (const uint4*)v_last_full, (const uint4*)x_e, slot, -dt_unedited, N, Ne_cap, (int)cpr,
+        (uint4*)x_out, dev_status));
 }

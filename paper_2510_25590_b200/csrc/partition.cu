@@ -113,6 +113,8 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
                  float threshold, uint8_t* __restrict__ mask, int32_t* __restrict__ edit_idx,
                  int32_t* __restrict__ keep_idx, int32_t* __restrict__ slot,
                  int32_t* __restrict__ n_edit, float* __restrict__ score) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     extern __shared__ uint32_t smem_u32[];
     const int nwords = share >> 5;
     uint32_t* bits = smem_u32;
@@ -274,6 +276,8 @@ __global__ void region_rows_kernel(const int32_t* __restrict__ edit_idx,
                                    int32_t* __restrict__ n_query, int q_cap,
                                    int32_t* __restrict__ cache_rows, int32_t* __restrict__ n_cache,
                                    int c_cap, int32_t* dev_status) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int b = blockIdx.y;
     int ne = n_edit[b];
     if (ne < 0 || ne > N) {
@@ -323,13 +327,15 @@ static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st
     cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)(share >> 5) * 8;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = csize;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see grid_dependency_wait
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, partition_kernel<L>, x_t, v, ref, N, C, share, t, metric, thr,
                               mask, edit_idx, keep_idx, slot, n_edit, score);
 }
@@ -405,8 +411,8 @@ extern "C" int regione_region_rows(const int32_t* edit_idx, const int32_t* keep_
     if (B == 0) return REGIONE_OK;
     const int span = (q_cap > c_cap ? q_cap : c_cap);
     dim3 grid((span + 255) / 256, B);
-    region_rows_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(
-        edit_idx, keep_idx, n_edit, N, n_text, n_ref, membership, query_rows, n_query, q_cap,
-        cache_rows, n_cache, c_cap, dev_status);
-    return launch_status(cudaGetLastError());
+    return launch_status(launch_overlapped(region_rows_kernel, grid, dim3(256), 0,
+                                           (cudaStream_t)stream, edit_idx, keep_idx, n_edit, N,
+                                           n_text, n_ref, membership, query_rows, n_query, q_cap,
+                                           cache_rows, n_cache, c_cap, dev_status));
 }

@@ -31,6 +31,8 @@ __global__ void __launch_bounds__(kCopyThreads)
 row_copy_kernel(const RowCopyPairs pairs, const int32_t* __restrict__ idx,
                 const int32_t* __restrict__ n, long long idx_rows, long long idx_stride,
                 long long cap, int cpr, int32_t* dev_status) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int b = blockIdx.y;
     const RowCopyPair p = pairs.p[blockIdx.z];
     long long live = n[b];
@@ -86,9 +88,9 @@ static int launch_row_copy(const RowCopyPairs& ps, int pairs, const int32_t* idx
     const long long blocks = (cap * cpr + per_block - 1) / per_block;
     if (cap * cpr + per_block >= 0x7fffffffLL) return REGIONE_UNSUPPORTED;
     dim3 grid((unsigned)blocks, (unsigned)B, (unsigned)pairs);
-    row_copy_kernel<GATHER><<<grid, kCopyThreads, 0, (cudaStream_t)stream>>>(
-        ps, idx, n, idx_rows, idx_stride, cap, (int)cpr, dev_status);
-    return launch_status(cudaGetLastError());
+    return launch_status(launch_overlapped(row_copy_kernel<GATHER>, grid, dim3(kCopyThreads), 0,
+                                           (cudaStream_t)stream, ps, idx, n, idx_rows, idx_stride,
+                                           cap, (int)cpr, dev_status));
 }
 
 }  // namespace regione

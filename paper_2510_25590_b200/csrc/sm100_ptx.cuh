@@ -206,15 +206,5 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, bool b_mn_ma
            | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Programmatic dependent launch.  `grid_launch_dependents` lets a kernel launched behind this one
-// with the programmatic-serialization attribute become resident early; `grid_dependency_wait` in
-// that kernel returns once the grid ahead of it has completed and its writes are visible.
-__device__ __forceinline__ void grid_launch_dependents() {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-__device__ __forceinline__ void grid_dependency_wait() {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-}
-
 }  // namespace ptx
 }  // namespace regione
