@@ -23,7 +23,10 @@
 // dependency chain of a tile (S -> softmax -> P*V -> next S) only stalls that
 // tile; the other tile's products fill the tensor pipe meanwhile.  The two
 // tiles take turns on the special-function unit (exp2), which keeps them out
-// of phase.
+// of phase.  A pair with a single live query tile does not leave the second
+// tile's warps idle: they run the same query tile against the odd key tiles of
+// the segment (own accumulator, maximum and sum in tensor memory / registers),
+// the first tile's warps take the even ones, and the epilogue merges the halves.
 //
 // Online softmax in the exp2 domain; O is rescaled in tensor memory only when
 // a row maximum grows by more than 2^8.  Keys past a segment's live count are
@@ -68,18 +71,23 @@ struct AttnCfg {
     static constexpr int kHalves = D / 64;
     static constexpr int kTileBytes = kHalves * kHalfBytes;
     static constexpr int kStages = (D == 128) ? 4 : 6;
-    static constexpr int kSmemTiles = (2 + kStages) * kTileBytes;
-    static constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 256 /*control*/;
+    // 2 query tiles + the ring + one more stage that only a lone query tile uses (its ring is that
+    // stage, the ordinary ring and the idle second query tile: kStages + 2 stages)
+    static constexpr int kSmemTiles = (2 + kStages + 1) * kTileBytes;
+    static constexpr int kCtrlBytes = 256;
+    static constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + kCtrlBytes +
+                                      kBM * 8 /*(max, sum) of a lone tile's second half*/;
 };
 
 struct AttnCtrl {
     uint64_t q_full;
-    uint64_t kv_full[6];
-    uint64_t kv_empty[6];
+    uint64_t kv_full[8];        // up to AttnCfg::kStages + 2 stages
+    uint64_t kv_empty[8];
     uint64_t s_full[2];         // [query tile]
     uint64_t p_full[2][2];      // [query tile][chunk of 64 keys]
     uint64_t o_final[2];        // completes once, after the tile's last P*V product
     uint64_t turn[2];           // turn[t]: the other query tile has finished a tile's exponentials
+    uint64_t half_done;         // lone query tile: the odd key tiles' (max, sum) are in shared memory
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -109,10 +117,10 @@ struct AttnParams {
 // ---- the plan every CTA (and the merge kernel) derives from the device-side counts ------------
 // Shares are cut on a cost axis measured in ticks, not in steps, so that they take about the same
 // time: a key tile of a full query pair costs kTickPair, a key tile of a pair with one live query
-// tile kTickSingle (it is bound by the tile's dependency chain, not by the work), and every item
-// starts with kTickStart ticks that stand for the drain of the previous segment and the fill of the
-// new one (measured on the kernel: 2.3 us, 2.0 us and about 8 us).
-constexpr int kTickPair = 8, kTickSingle = 7, kTickStart = 28;
+// tile kTickSingle (its even and odd key tiles run side by side on the two tile roles, so it costs
+// a little more than half as much), and every item starts with kTickStart ticks that stand for the
+// drain of the previous segment and the fill of the new one (measured on the kernel).
+constexpr int kTickPair = 8, kTickSingle = 5, kTickStart = 28;
 
 struct ReqShape {
     int nq, nf, nc;      // clamped counts
@@ -278,16 +286,21 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
-// Maximum of 64 logits held in registers (keys >= valid masked out).
-template <bool MASK>
-__device__ __forceinline__ float chunk_max(const uint32_t* s, int valid) {
+// Keys >= valid of a 64-logit chunk are dead (behind a segment's live prefix): their logits become
+// -inf, after which the chunk goes through the same code as a full one (maximum unaffected,
+// probability 0 or, on the polynomial path, 2^-126).  A short separate pass instead of masked
+// variants of the long unrolled loops: those would run once per item, from a cold instruction cache.
+__device__ __forceinline__ void mask_dead_keys(uint32_t* s, int valid) {
+#pragma unroll
+    for (int i = 0; i < kBH; ++i)
+        if (i >= valid) s[i] = 0xff800000u;
+}
+
+// Maximum of 64 logits held in registers.
+__device__ __forceinline__ float chunk_max(const uint32_t* s) {
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-    for (int i = 0; i < kBH; ++i) {
-        float v = __uint_as_float(s[i]);
-        if (MASK && i >= valid) v = -INFINITY;
-        mx[i & 3] = fmaxf(mx[i & 3], v);
-    }
+    for (int i = 0; i < kBH; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(s[i]));
     return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 }
 
@@ -307,18 +320,14 @@ __device__ __forceinline__ float poly_exp2(float x) {
 
 // p = 2^(s*c - m) for 64 logits, written to tensor memory at `tP` (32 columns) as packed bf16;
 // returns their fp32 sum.
-template <bool MASK>
-__device__ __forceinline__ float chunk_probabilities(uint32_t tP, const uint32_t* s, int valid,
-                                                     float c, float m) {
+__device__ __forceinline__ float chunk_probabilities(uint32_t tP, const uint32_t* s, float c, float m) {
     float sum[4] = {0.f, 0.f, 0.f, 0.f};
     uint32_t pk[kBH / 2];
 #pragma unroll
     for (int i = 0; i < kBH / 2; ++i) {
-        float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, -m));
-        float p1 = (i % kPolyEvery == 0) ? poly_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m))
-                                         : fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m));
-        if (MASK && 2 * i >= valid) p0 = 0.f;
-        if (MASK && 2 * i + 1 >= valid) p1 = 0.f;
+        const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, -m));
+        const float p1 = (i % kPolyEvery == 0) ? poly_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m))
+                                               : fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m));
         sum[i & 3] += p0 + p1;
         pk[i] = pack_bf16x2(p0, p1);
     }
@@ -372,12 +381,23 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     // slot of this segment among the shares that touch the item; a lone segment writes the output
     const int slot = it.slot;
     const bool direct = it.n_slots == 1;
+    // A lone query tile would leave half of the CTA idle and run at the speed of its dependency
+    // chain.  Instead the roles of "tile 1" work on the same query tile against the odd key tiles
+    // of the segment while "tile 0" takes the even ones; the two halves (own accumulator, maximum
+    // and sum) are merged in the epilogue.  `lanes` = query-tile roles at work.
+    const bool split = ntq == 1 && n_tiles >= 2;
+    const int lanes = split ? 2 : ntq;
+    // a lone tile's ring starts at the idle second query tile and runs over the extra stage: two
+    // stages more, because its two halves consume K/V tiles at twice the rate per chain
+    const int n_stages = split ? kStages + 2 : kStages;
+    const uint32_t ring = split ? sQ + kTileBytes : sKV;
+    uint8_t* const ring_gen = smem_gen + (split ? 1 : 2) * kTileBytes;
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(ptx::smem_addr(&ctrl->q_full), 1);
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kStages + 2; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctrl->kv_full[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_empty[s]), ntq);    // one commit per issuer
+            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_empty[s]), split ? 1 : ntq);   // commits per stage
         }
         for (int t = 0; t < 2; ++t) {
             ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t]), 1);
@@ -386,6 +406,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             ptx::mbar_init(ptx::smem_addr(&ctrl->o_final[t]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctrl->turn[t]), kBM / 32);
         }
+        ptx::mbar_init(ptx::smem_addr(&ctrl->half_done), kBM / 32);
         ptx::fence_barrier_init();
     }
     ptx::tc_fence_before_sync();
@@ -407,6 +428,9 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         tile_seg(jl, cached, row0, valid);
         return valid > kBH ? 2 : 1;
     };
+    // key tiles of query-tile role t: all of them, or every second one of a lone query tile
+    auto role_tiles = [&](int t) { return split ? (n_tiles + 1 - t) >> 1 : n_tiles; };
+    auto role_tile = [&](int t, int j) { return split ? 2 * j + t : j; };
 
     if constexpr (!SOFTMAX_WG) {
     if (warp == 8) {
@@ -424,7 +448,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             bool ok = true;
             for (int i = 0; i < 2 * n_tiles && ok; ++i) {
                 const int j = i >> 1, is_v = i & 1;
-                const int stage = i % kStages, use = i / kStages;
+                const int stage = i % n_stages, use = i / n_stages;
                 if (use > 0)
                     ok = wait_bar(ptx::smem_addr(&ctrl->kv_empty[stage]), (use - 1) & 1, abort_flag,
                                   p.dev_status);
@@ -435,7 +459,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 const uint32_t bar = ptx::smem_addr(&ctrl->kv_full[stage]);
                 ptx::mbar_arrive_expect_tx(bar, kTileBytes);
                 for (int hf = 0; hf < Cfg::kHalves; ++hf)
-                    ptx::tma_load_4d(sKV + stage * kTileBytes + hf * kHalfBytes, map, bar, hf * 64, h,
+                    ptx::tma_load_4d(ring + stage * kTileBytes + hf * kHalfBytes, map, bar, hf * 64, h,
                                      row0, b);
             }
         }
@@ -443,15 +467,16 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         // ================= MMA issuers: warp 9 for query tile 0, warp 10 for query tile 1 ========
         // Each whole warp walks its loop and waits on the barriers; one elected lane issues.
         const int t = warp - 9;
-        if (t < ntq && n_tiles > 0) {
+        if (t < lanes && n_tiles > 0) {
+            const int n_my = role_tiles(t);
             constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
             constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
             // K-major operands (Q, K): 128-byte swizzle, LBO unused; V is MN-major: 64-column
             // boxes kHalfBytes apart (LBO), 8-key groups 1024 B apart (SBO).
-            const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
-            const uint32_t k_lo = ptx::smem_desc_lo(sKV, 16);
-            const uint32_t v_lo = ptx::smem_desc_lo(sKV, kHalfBytes);
+            const uint32_t q_lo = ptx::smem_desc_lo(sQ + (split ? 0 : t) * kTileBytes, 16);
+            const uint32_t k_lo = ptx::smem_desc_lo(ring, 16);
+            const uint32_t v_lo = ptx::smem_desc_lo(ring, kHalfBytes);
             const uint32_t tSt = tmem + t * kBN, tOt = tmem + 256 + t * D;
             // S_t = Q_t K^T
             auto issue_s = [&](int stage) {
@@ -474,25 +499,28 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                                 (accumulate || kk > 0) ? 1u : 0u);
             };
             bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
-            if (ok && n_tiles > 0) {
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[0]), 0, abort_flag, p.dev_status);
+            if (ok) {
+                const int ik0 = 2 * role_tile(t, 0), sk0 = ik0 % n_stages;
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk0]), (ik0 / n_stages) & 1, abort_flag,
+                              p.dev_status);
                 if (ok) {
                     ptx::tc_fence_after_sync();
                     if (ptx::elect_one()) {
-                        issue_s(0);
+                        issue_s(sk0);
                         ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[0]));
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk0]));
                     }
                     __syncwarp();
                 }
             }
             int nb = 0;                                     // second chunks seen so far
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int iv = 2 * j + 1, ik = 2 * j + 2;
-                const int sv = iv % kStages, sk = ik % kStages;
-                const bool more = (j + 1 < n_tiles);
-                const int chunks = tile_chunks(j);
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+            for (int j = 0; j < n_my && ok; ++j) {
+                const int jl = role_tile(t, j);
+                const int iv = 2 * jl + 1, ik = 2 * role_tile(t, j + 1);
+                const int sv = iv % n_stages, sk = ik % n_stages;
+                const bool more = (j + 1 < n_my);
+                const int chunks = tile_chunks(jl);
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / n_stages) & 1, abort_flag,
                               p.dev_status);
                 if (ok)
                     ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][0]), j & 1, abort_flag,
@@ -504,7 +532,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                     __syncwarp();
                 }
                 if (more)
-                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / kStages) & 1, abort_flag,
+                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / n_stages) & 1, abort_flag,
                                   p.dev_status);
                 if (ok && chunks == 2) {
                     ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][1]), nb & 1, abort_flag,
@@ -527,7 +555,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             }
         }
     }
-    } else if (warp < 4 * ntq) {
+    } else if (warp < 4 * lanes) {
         // ================= softmax / correction / epilogue =================
         const int t = warp >> 2;
         const int row = ((warp & 3) << 5) + lane;                  // row of the query tile
@@ -537,9 +565,10 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_tiles; ++j) {
+        const int n_my = n_tiles > 0 ? role_tiles(t) : 0;
+        for (int j = 0; j < n_my; ++j) {
             bool cached; int row0, valid;
-            tile_seg(j, cached, row0, valid);
+            tile_seg(role_tile(t, j), cached, row0, valid);
             const int chunks = valid > kBH ? 2 : 1;
             ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status);
             if (!ok) break;
@@ -554,12 +583,13 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             if (chunks == 2) {
                 ptx::tmem_ld32(tS + 64, s + 64);
                 ptx::tmem_ld32(tS + 96, s + 96);
-                mt = chunk_max<false>(s, kBH);
+                mt = chunk_max(s);
                 ptx::tmem_wait_ld();
-                mt = fmaxf(mt, valid == kBN ? chunk_max<false>(s + kBH, kBH)
-                                            : chunk_max<true>(s + kBH, valid - kBH));
+                if (valid < kBN) mask_dead_keys(s + kBH, valid - kBH);
+                mt = fmaxf(mt, chunk_max(s + kBH));
             } else {
-                mt = valid == kBH ? chunk_max<false>(s, kBH) : chunk_max<true>(s, valid);
+                if (valid < kBH) mask_dead_keys(s, valid);
+                mt = chunk_max(s);
             }
             mt *= c;
             if (j == 0) {
@@ -584,25 +614,24 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             // tile j + 1 after tile 1 has finished j.  Run alone they take half as long, which
             // shortens each tile's chain S -> softmax -> P*V -> next S; the other tile's loads,
             // maxima and products fall into the gap.
-            if (ntq == 2 && (t == 1 || j > 0)) {
+            if (lanes == 2 && (t == 1 || j > 0)) {
                 ok = wait_bar(ptx::smem_addr(&ctrl->turn[t]), (j - 1 + t) & 1, abort_flag,
                               p.dev_status);
                 if (!ok) break;
             }
             // first chunk of probabilities (keys 0..63 of the tile)
-            l += (valid >= kBH) ? chunk_probabilities<false>(tS, s, kBH, c, m)
-                                : chunk_probabilities<true>(tS, s, valid, c, m);
-            if (chunks == 1 && ntq == 2 && lane == 0)
+            l += chunk_probabilities(tS, s, c, m);
+            if (chunks == 1 && lanes == 2 && lane == 0)
                 ptx::mbar_arrive(ptx::smem_addr(&ctrl->turn[t ^ 1]));
             ptx::tmem_wait_st();
             if (valid < kBN) {
                 // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
-                const int iv = 2 * j + 1, sv = iv % kStages;
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / kStages) & 1, abort_flag,
+                const int iv = 2 * role_tile(t, j) + 1, sv = iv % n_stages;
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / n_stages) & 1, abort_flag,
                               p.dev_status);
                 if (!ok) break;
                 if (row >= valid) {
-                    uint8_t* vrow = smem_gen + 2 * kTileBytes + sv * kTileBytes + row * 128;
+                    uint8_t* vrow = ring_gen + sv * kTileBytes + row * 128;
 #pragma unroll
                     for (int hf = 0; hf < Cfg::kHalves; ++hf)
 #pragma unroll
@@ -616,9 +645,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t][0]));
             if (chunks == 2) {
                 // second chunk (keys 64..127) while the first chunk's product runs
-                l += (valid == kBN) ? chunk_probabilities<false>(tS + kBH / 2, s + kBH, kBH, c, m)
-                                    : chunk_probabilities<true>(tS + kBH / 2, s + kBH, valid - kBH, c, m);
-                if (ntq == 2 && lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->turn[t ^ 1]));
+                l += chunk_probabilities(tS + kBH / 2, s + kBH, c, m);
+                if (lanes == 2 && lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->turn[t ^ 1]));
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
@@ -629,13 +657,45 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         // from registers would touch 32 different rows per warp instruction; instead each warp
         // passes 128-byte row pieces through its own 4 KB corner of the (now idle) query tile in
         // shared memory and stores four whole pieces per instruction.
-        const int wrow0 = q0 + t * kBM + ((warp & 3) << 5);         // first query row of this warp
+        const int wrow0 = q0 + (split ? 0 : t) * kBM + ((warp & 3) << 5);   // first query row of this warp
         const int live_rows = min(max(nq - wrow0, 0), 32);
         const bool live = lane < live_rows;
         if (n_tiles > 0 && ok) {
             ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status);
             if (ok) ptx::tc_fence_after_sync();
         }
+        // lone query tile: role 1 leaves its (max, sum) in shared memory (its accumulator stays in
+        // tensor memory) and is done; role 0 merges the halves
+        float2* const half_ml = reinterpret_cast<float2*>(smem_gen + Cfg::kSmemTiles + Cfg::kCtrlBytes);
+        float w_own = 1.f, w_other = 0.f;                   // weights of the two accumulators
+        if (split && t == 1) {
+            half_ml[row] = make_float2(m, l);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->half_done));
+        } else if (split && ok) {
+            ok = wait_bar(ptx::smem_addr(&ctrl->half_done), 0, abort_flag, p.dev_status);
+            if (ok) ok = wait_bar(ptx::smem_addr(&ctrl->o_final[1]), 0, abort_flag, p.dev_status);
+            if (ok) {
+                ptx::tc_fence_after_sync();
+                const float2 other = half_ml[row];
+                const float m_all = fmaxf(m, other.x);
+                w_own = fast_exp2(m - m_all);
+                w_other = other.y > 0.f ? fast_exp2(other.x - m_all) : 0.f;
+                l = w_own * l + w_other * other.y;
+                m = m_all;
+            }
+        }
+        // lone tile: 32 columns of this row's two accumulators, weighted and added
+        auto load_merged = [&](int col, uint32_t* r) {
+            uint32_t r1[32];
+            ptx::tmem_ld32(tO + col, r);
+            ptx::tmem_ld32(tO + D + col, r1);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                r[i] = __float_as_uint(fmaf(w_own, __uint_as_float(r[i]), w_other * __uint_as_float(r1[i])));
+        };
+        if (!(split && t == 1)) {
         uint8_t* const stage = smem_gen + t * kTileBytes + (warp & 3) * (kTileBytes / 4);
         auto store_pieces = [&](const uint4 (&v)[8], uint8_t* g_row0, size_t row_stride) {
             // piece q of row r sits at 16-byte column q ^ (r & 7): both the row-wise writes and
@@ -668,9 +728,14 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
 #pragma unroll 1
                 for (int c64 = 0; c64 < D / 64; ++c64) {
                     uint32_t r[64];
-                    ptx::tmem_ld32(tO + c64 * 64, r);
-                    ptx::tmem_ld32(tO + c64 * 64 + 32, r + 32);
-                    ptx::tmem_wait_ld();
+                    if (!split) {
+                        ptx::tmem_ld32(tO + c64 * 64, r);
+                        ptx::tmem_ld32(tO + c64 * 64 + 32, r + 32);
+                        ptx::tmem_wait_ld();
+                    } else {
+                        load_merged(c64 * 64, r);
+                        load_merged(c64 * 64 + 32, r + 32);
+                    }
                     uint4 v[8];
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
@@ -685,7 +750,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         } else {
             // unnormalised O and (m, l) of this segment -> its workspace slot
             const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + it.qp;
-            const size_t prow_w = (item_idx * p.max_slots + slot) * (2 * kBM) + t * kBM + ((warp & 3) << 5);
+            const size_t prow_w = (item_idx * p.max_slots + slot) * (2 * kBM) + (split ? 0 : t) * kBM +
+                                  ((warp & 3) << 5);
             if (n_tiles == 0) {
                 if (live) p.part_ml[prow_w + lane] = make_float2(-INFINITY, 0.f);
             } else if (ok) {
@@ -693,8 +759,12 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
 #pragma unroll 1
                 for (int ch = 0; ch < D / 32; ++ch) {
                     uint32_t r[32];
-                    ptx::tmem_ld32(tO + ch * 32, r);
-                    ptx::tmem_wait_ld();
+                    if (!split) {
+                        ptx::tmem_ld32(tO + ch * 32, r);
+                        ptx::tmem_wait_ld();
+                    } else {
+                        load_merged(ch * 32, r);
+                    }
                     uint4 v[8];
 #pragma unroll
                     for (int q = 0; q < 8; ++q) v[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
@@ -703,6 +773,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 if (live) p.part_ml[prow_w + lane] = make_float2(m, l);
             }
         }
+        }   // all roles but the second half of a lone tile
         ptx::fence_proxy_async_smem();      // the next segment's query tile arrives by TMA
     }
 
@@ -712,7 +783,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     ptx::tc_fence_after_sync();
     if (threadIdx.x == 0) {
         ptx::mbar_inval(ptx::smem_addr(&ctrl->q_full));
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kStages + 2; ++s) {
             ptx::mbar_inval(ptx::smem_addr(&ctrl->kv_full[s]));
             ptx::mbar_inval(ptx::smem_addr(&ctrl->kv_empty[s]));
         }
@@ -723,6 +794,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             ptx::mbar_inval(ptx::smem_addr(&ctrl->o_final[t]));
             ptx::mbar_inval(ptx::smem_addr(&ctrl->turn[t]));
         }
+        ptx::mbar_inval(ptx::smem_addr(&ctrl->half_done));
     }
     pos = pl.whole_items ? pos + gridDim.x : it.next;
     if (*abort_flag) break;
