@@ -49,6 +49,7 @@
 // records REGIONE_DEV_TIMEOUT, all roles leave their loops, tensor memory is
 // released and the kernel ends normally.
 #include <cuda.h>
+#include <cstddef>
 #include <type_traits>
 
 #include <algorithm>
@@ -91,6 +92,13 @@ struct AttnCtrl {
     uint32_t tmem_base;
     int abort_flag;
 };
+
+// The barriers of AttnCtrl as one array starting at q_full.
+constexpr int kBarKvEmpty = 9, kBarSFull = 17, kBarPFull = 19, kBarOFinal = 23, kBarTurn = 25, kNumBarriers = 28;
+static_assert(offsetof(AttnCtrl, kv_empty) == kBarKvEmpty * 8 && offsetof(AttnCtrl, s_full) == kBarSFull * 8 &&
+              offsetof(AttnCtrl, p_full) == kBarPFull * 8 && offsetof(AttnCtrl, o_final) == kBarOFinal * 8 &&
+              offsetof(AttnCtrl, turn) == kBarTurn * 8 && offsetof(AttnCtrl, tmem_base) == kNumBarriers * 8,
+              "barrier layout");
 
 // What share c tells the merge kernel: the item that the boundary between shares c - 1 and c
 // cuts, if c is the second share of that item (so every cut item is named exactly once).
@@ -393,20 +401,13 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     const uint32_t ring = split ? sQ + kTileBytes : sKV;
     uint8_t* const ring_gen = smem_gen + (split ? 1 : 2) * kTileBytes;
 
-    if (threadIdx.x == 0) {
-        ptx::mbar_init(ptx::smem_addr(&ctrl->q_full), 1);
-        for (int s = 0; s < kStages + 2; ++s) {
-            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_full[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->kv_empty[s]), split ? 1 : ntq);   // commits per stage
-        }
-        for (int t = 0; t < 2; ++t) {
-            ptx::mbar_init(ptx::smem_addr(&ctrl->s_full[t]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t][0]), kBM / 32);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->p_full[t][1]), kBM / 32);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->o_final[t]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctrl->turn[t]), kBM / 32);
-        }
-        ptx::mbar_init(ptx::smem_addr(&ctrl->half_done), kBM / 32);
+    // thread i sets barrier i of the control block up (and takes it down after the segment)
+    if (threadIdx.x < kNumBarriers) {
+        const int i = threadIdx.x;
+        int count = 1;                                               // q_full, kv_full, s_full, o_final
+        if (i >= kBarKvEmpty && i < kBarSFull) count = split ? 1 : ntq;             // commits per stage
+        else if ((i >= kBarPFull && i < kBarOFinal) || i >= kBarTurn) count = kBM / 32;   // one arrival per warp
+        ptx::mbar_init(ptx::smem_addr(&ctrl->q_full + i), count);
         ptx::fence_barrier_init();
     }
     ptx::tc_fence_before_sync();
@@ -781,21 +782,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
-    if (threadIdx.x == 0) {
-        ptx::mbar_inval(ptx::smem_addr(&ctrl->q_full));
-        for (int s = 0; s < kStages + 2; ++s) {
-            ptx::mbar_inval(ptx::smem_addr(&ctrl->kv_full[s]));
-            ptx::mbar_inval(ptx::smem_addr(&ctrl->kv_empty[s]));
-        }
-        for (int t = 0; t < 2; ++t) {
-            ptx::mbar_inval(ptx::smem_addr(&ctrl->s_full[t]));
-            ptx::mbar_inval(ptx::smem_addr(&ctrl->p_full[t][0]));
-            ptx::mbar_inval(ptx::smem_addr(&ctrl->p_full[t][1]));
-            ptx::mbar_inval(ptx::smem_addr(&ctrl->o_final[t]));
-            ptx::mbar_inval(ptx::smem_addr(&ctrl->turn[t]));
-        }
-        ptx::mbar_inval(ptx::smem_addr(&ctrl->half_done));
-    }
+    if (threadIdx.x < kNumBarriers) ptx::mbar_inval(ptx::smem_addr(&ctrl->q_full + threadIdx.x));
     pos = pl.whole_items ? pos + gridDim.x : it.next;
     if (*abort_flag) break;
     }   // segments
