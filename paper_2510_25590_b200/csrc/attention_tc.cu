@@ -209,11 +209,19 @@ struct Segment {
     long long next;         // position behind the item
 };
 
+// a / b for non-negative a and positive b; positions fit 32 bits in every realistic launch, and a
+// 32-bit division is several times shorter than a 64-bit one (the lookups below sit between two
+// segments, on every thread's path).
+__device__ __forceinline__ long long div_pos(long long a, long long b) {
+    if (((a | b) >> 32) == 0) return (long long)((unsigned)a / (unsigned)b);
+    return a / b;
+}
+
 // Shares that hold steps of the item whose step 0 starts at tick `first_tick`.
 __device__ __forceinline__ void item_slots(const Plan& pl, long long first_tick, int w, int steps,
                                            int& c_first, int& n_slots) {
-    c_first = (int)(first_tick / pl.chunk);
-    n_slots = (int)((first_tick + (long long)w * (steps - 1)) / pl.chunk) - c_first + 1;
+    c_first = (int)div_pos(first_tick, pl.chunk);
+    n_slots = (int)div_pos(first_tick + (long long)w * (steps - 1), pl.chunk) - c_first + 1;
 }
 
 // Whole-item plan: the item with index `idx`.
@@ -258,16 +266,16 @@ __device__ __forceinline__ Segment segment_ticks(const AttnParams& p, const Plan
         return sg;
     }
     const long long rel = pos - base;
-    sg.h = (int)(rel / r.head_ticks);
+    sg.h = (int)div_pos(rel, r.head_ticks);
     const long long rem = rel - (long long)sg.h * r.head_ticks;
-    sg.qp = (int)min(rem / r.ticks_full, (long long)(r.np - 1));
+    sg.qp = (int)min(div_pos(rem, r.ticks_full), (long long)(r.np - 1));
     const long long t0 = base + (long long)sg.h * r.head_ticks + (long long)sg.qp * r.ticks_full;
     const bool last = sg.qp == r.np - 1;
     const int w = last ? r.w_last : kTickPair;
     const long long first_tick = t0 + kTickStart;
     const long long lo = (long long)c * pl.chunk, hi = lo + pl.chunk;
-    long long s_lo = lo <= first_tick ? 0 : (lo - first_tick + w - 1) / w;
-    long long s_hi = hi <= first_tick ? 0 : (hi - first_tick + w - 1) / w;
+    long long s_lo = lo <= first_tick ? 0 : div_pos(lo - first_tick + w - 1, w);
+    long long s_hi = hi <= first_tick ? 0 : div_pos(hi - first_tick + w - 1, w);
     s_lo = min(s_lo, (long long)r.steps);
     s_hi = min(s_hi, (long long)r.steps);
     sg.j_first = (int)s_lo;
