@@ -126,9 +126,9 @@ struct AttnParams {
 // Shares are cut on a cost axis measured in ticks, not in steps, so that they take about the same
 // time: a key tile of a full query pair costs kTickPair, a key tile of a pair with one live query
 // tile kTickSingle (its even and odd key tiles run side by side on the two tile roles, so it costs
-// a little more than half as much), and every item starts with kTickStart ticks that stand for the
+// half as much), and every item starts with kTickStart ticks that stand for the
 // drain of the previous segment and the fill of the new one (measured on the kernel).
-constexpr int kTickPair = 8, kTickSingle = 5, kTickStart = 28;
+constexpr int kTickPair = 8, kTickSingle = 4, kTickStart = 28;
 
 struct ReqShape {
     int nq, nf, nc;      // clamped counts
