@@ -867,11 +867,12 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
 // is launched behind the attention kernel with programmatic serialization and reads nothing before
 // the dependency wait; all slots' loads are issued before the first use, so a warp pays one
 // memory round trip, not one per slot.
-constexpr int kCombineMaxSlots = 8;      // upper bound of AttnParams::max_slots
-
-template <int D>
+// MAXS >= AttnParams::max_slots bounds the slots held in registers (the host knows max_slots, and
+// the smaller instantiations let more warps be resident).
+template <int D, int MAXS>
 __global__ void __launch_bounds__(256)
 region_attention_combine_kernel(const AttnParams p) {
+    constexpr int kCombineMaxSlots = MAXS;
     constexpr int E = D / 32;
     using Vec = typename std::conditional<E == 4, float4, float2>::type;
     grid_dependency_wait();
@@ -1024,10 +1025,17 @@ static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, c
     // the merge kernel may become resident while the attention kernel drains (it waits for that
     // kernel's completion before it reads a slot)
     if (grid < 2) return launch_status(cudaGetLastError());     // a single share cuts nothing
-    if (launch_overlapped(region_attention_combine_kernel<D>,
-                          dim3((unsigned)(grid - 1), (2 * kBM) / 8, 1), dim3(256), 0, st,
-                          prm) != cudaSuccess)
-        return REGIONE_CUDA_ERROR;
+    const dim3 cgrid((unsigned)(grid - 1), (2 * kBM) / 8, 1);
+    cudaError_t e;
+    if (prm.max_slots <= 2)
+        e = launch_overlapped(region_attention_combine_kernel<D, 2>, cgrid, dim3(256), 0, st, prm);
+    else if (prm.max_slots <= 3)
+        e = launch_overlapped(region_attention_combine_kernel<D, 3>, cgrid, dim3(256), 0, st, prm);
+    else if (prm.max_slots <= 4)
+        e = launch_overlapped(region_attention_combine_kernel<D, 4>, cgrid, dim3(256), 0, st, prm);
+    else
+        e = launch_overlapped(region_attention_combine_kernel<D, 8>, cgrid, dim3(256), 0, st, prm);
+    if (e != cudaSuccess) return REGIONE_CUDA_ERROR;
     return launch_status(cudaGetLastError());
 }
 
