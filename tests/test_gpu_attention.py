@@ -213,6 +213,35 @@ def test_tensor_core_kernel_agrees_with_cuda_core_kernel_on_every_row():
     want = orc.region_attention(c["q"], c["kf"], c["vf"], c["kc"], c["vc"], c["nq"], c["nf"], c["nc"])
     assert_close(s, want, "cuda-core kernel vs oracle")
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("counts", [
+    # a lone query tile against an odd and an even number of key tiles (its key tiles are dealt to both
+    # tile roles alternately and the halves merged), ragged ends in both segments
+    [(100, 100, 647)],
+    [(128, 128, 896)],
+    [(51, 51, 2 * 128 + 1)],
+    # pairs followed by a lone last tile, shares cutting items of both kinds
+    [(300, 300, 2000)],
+    # requests of different shapes in one launch, one of them empty
+    [(330, 330, 1500), (77, 77, 900), (256, 256, 1200), (0, 10, 10)],
+    # query count a multiple of 128 but not of 256; no fresh keys at all
+    [(384, 0, 1100)],
+])
+def test_every_row_under_mixed_plans(counts, D):
+    """Every output row against the oracle on shapes that mix full pairs, lone tiles and cut items."""
+    B, H = len(counts), 3
+    cap_q = max(c[0] for c in counts) + 1
+    cap_f = max(max(c[1] for c in counts), 1)
+    cap_c = max(c[2] for c in counts) + 3
+    rng = np.random.default_rng(sum(sum(c) for c in counts) + D)
+    q = _rand_bf16(rng, (B, cap_q, H, D), 0.5)
+    kf, vf = _rand_bf16(rng, (B, cap_f, H, D), 0.5), _rand_bf16(rng, (B, cap_f, H, D))
+    kc, vc = _rand_bf16(rng, (B, cap_c, H, D), 0.5), _rand_bf16(rng, (B, cap_c, H, D))
+    n_q = np.array([c[0] for c in counts], np.int32)
+    n_f = np.array([c[1] for c in counts], np.int32)
+    n_c = np.array([c[2] for c in counts], np.int32)
+    check(q, kf, vf, kc, vc, n_q, n_f, n_c, what=f"mixed plans {counts} D={D}")
+
 
 @pytest.mark.parametrize("caps,counts", [
     # capacities far above the live counts: the plan comes from the device-side counts, the workspace
