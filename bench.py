@@ -215,13 +215,26 @@ def hbm_sweep(torch, binding, step, d, flush_l2, peak_gbs, iters=10):
     n_cache = int(step.n_cache.sum().item())
     timed("rikv_store (bench workload)", n_cache * (4 * row + 4),
           lambda: binding.rikv_store(d["k"], d["vv"], step.cache_rows, step.n_cache, step.k_cache, step.v_cache))
-    rows = 16384                                            # 100 MB read + 100 MB written
-    idx = (torch.arange(rows, device="cuda", dtype=i32) * 7 % d["k"].shape[1]).sort()[0].to(i32).reshape(1, rows)
-    idx = idx.expand(d["k"].shape[0], rows).contiguous()
-    n_rows = torch.full((d["k"].shape[0],), rows, dtype=i32, device="cuda")
-    dst = torch.empty((d["k"].shape[0], rows, s.H, s.D), dtype=bf, device="cuda")
-    timed("gather of 16384 rows of 6 KB", d["k"].shape[0] * rows * (2 * row + 4),
-          lambda: binding.gather(d["k"], idx, n_rows, dst))
+    # the same store at config 5's size (4 requests, 17562 of 18944 rows kept each): 1.7 GB, long enough
+    # that the ramp and the tail of the launch no longer count
+    gs5 = torch.Generator(device="cuda"); gs5.manual_seed(12)
+    k5 = torch.empty((4, 18944, s.H, s.D), dtype=bf, device="cuda").normal_(generator=gs5)
+    v5 = torch.empty((4, 18944, s.H, s.D), dtype=bf, device="cuda").normal_(generator=gs5)
+    keep5 = torch.stack([torch.randperm(18944, device="cuda", generator=gs5)[:17562].sort()[0] for _ in range(4)]).to(i32).contiguous()
+    n5 = torch.full((4,), 17562, dtype=i32, device="cuda")
+    kc5 = torch.empty((4, 17562, s.H, s.D), dtype=bf, device="cuda"); vc5 = torch.empty_like(kc5)
+    timed("rikv_store (config 5's size)", 4 * 17562 * (4 * row + 4),
+          lambda: binding.rikv_store(k5, v5, keep5, n5, kc5, vc5))
+    del k5, v5, kc5, vc5
+    rows, src_rows = 16384, 32768                           # 100 MB read + 100 MB written, every row once
+    gs = torch.Generator(device="cuda"); gs.manual_seed(11)
+    src = torch.empty((1, src_rows, s.H, s.D), dtype=bf, device="cuda").normal_(generator=gs)
+    idx = torch.randperm(src_rows, device="cuda", generator=gs)[:rows].sort()[0].to(i32).reshape(1, rows).contiguous()
+    n_rows = torch.full((1,), rows, dtype=i32, device="cuda")
+    dst = torch.empty((1, rows, s.H, s.D), dtype=bf, device="cuda")
+    timed("gather of 16384 distinct rows of 6 KB", rows * (2 * row + 4),
+          lambda: binding.gather(src, idx, n_rows, dst))
+    del src, dst
     B, N, C = 32, 65536, 16
     g = torch.Generator(device="cuda"); g.manual_seed(7)
     ref = torch.randn((B, N, C), device="cuda", generator=g).to(bf)
