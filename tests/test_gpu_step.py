@@ -66,3 +66,41 @@ def test_config4_shape_small_l2_metric():
 
 def test_zero_edit_mask_is_one_step_prediction_everywhere():
     run_step(synth.scaled_workload(synth.WORKLOADS[2], grid=(16, 16), n_text=16, heads=2), ratio=0.0)
+
+
+def test_step_replayed_from_a_cuda_graph_matches_the_eager_step():
+    """The ten launches of a step (each with programmatic stream serialization) captured into a
+    CUDA graph and replayed give bit-identical buffers to the same step launched eagerly."""
+    import torch
+    wl = synth.scaled_workload(synth.WORKLOADS[2], grid=(24, 24), n_text=70)
+    lat = synth.make_latents(wl)
+    qkv = synth.make_qkv_full(wl)
+    t, scale, dt, dt_u = lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0
+    d = {k: dev_bf16(lat[k]) for k in ("x_t", "v", "ref")}
+    dq, dk, dv = (dev_bf16(qkv[k]) for k in ("q", "k", "v"))
+    cap = plan_capacity(d["x_t"], d["v"], d["ref"], t, binding.METRIC_COSINE, wl.threshold)
+    shp = StepShapes(wl.batch, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads, wl.head_dim, cap,
+                     binding.METRIC_COSINE, wl.threshold, binding.ROWS_EDITED_QUERIES)
+    step = RegionStep(shp)
+    names = ("mask", "slot", "n_edit", "k_cache", "v_cache", "o_e", "o_full", "x_e", "x_out")
+    def run():
+        step.run(d["x_t"], d["v"], d["ref"], dq, dk, dv, t, scale, dt, dt_u)
+    step.o_full.fill_(0)
+    run()                                   # eager (also the first-call set-up, outside any capture)
+    torch.cuda.synchronize()
+    eager = {n: getattr(step, n).clone() for n in names}
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            run()
+    for n in names:
+        getattr(step, n).zero_()
+    torch.cuda.synchronize()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(step.dev_status[0]) == 0
+    for n in names:
+        a, b = eager[n], getattr(step, n)
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), n
