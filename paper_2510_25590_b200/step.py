@@ -4,9 +4,11 @@ This is call sequencing and buffer ownership only (torch tensors are device
 buffers): every operation runs in the library's kernels.  The sequence follows
 Algorithm 1 of the paper for one layer:
 
-  partition -> row lists -> gather X^E, v^E (one launch) -> RIKV store -> gather Q/K/V of the
-  recomputed rows (one launch) -> region attention -> scatter the attention rows back ->
-  velocity decay + Euler update -> merge with one-step-predicted unedited tokens.
+  partition -> row lists -> two independent branches, joined before the step returns:
+    attention branch: RIKV store -> gather Q/K/V of the recomputed rows (one launch) ->
+                      region attention -> scatter the attention rows back
+    latent branch   : gather X^E, v^E (one launch) -> velocity decay + Euler update -> merge with
+                      the one-step-predicted unedited tokens (on a side stream)
 
 No step needs a host round trip: per-request counts stay in device memory.
 Capacities are host integers chosen by the caller (``plan_capacity`` reads the
@@ -82,9 +84,12 @@ class RegionStep:
         ws = binding.region_attention_workspace(B, shp.q_cap, shp.q_cap, shp.c_cap, H, D)
         self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=device)
         self.launches = 0
+        self._side = torch.cuda.Stream(device=device)
+        self._fork, self._join = torch.cuda.Event(), torch.cuda.Event()
         self.attention_events = None      # optional (start, stop) pair recorded around the attention
 
     def run(self, x_t, v, ref, q_full, k_full, v_full, t, scale, dt, dt_unedited, stream=None):
+        import torch
         s = self.shp
         st = self.dev_status
         b = binding
@@ -93,8 +98,20 @@ class RegionStep:
         b.region_rows(self.edit_idx, self.keep_idx, self.n_edit, s.n_text, s.n_ref, s.membership,
                       self.query_rows, self.n_q, self.cache_rows, self.n_cache, dev_status=st,
                       stream=stream)
+        # Two independent branches hang off the partition: the latent branch (gather of X^E and v,
+        # velocity decay, merge: small latency-bound kernels) and the attention branch (cache store,
+        # gather of Q/K/V, attention, scatter).  The latent branch runs on a side stream so that it
+        # falls into the shadow of the cache store; both join before the step returns.
+        main = torch.cuda.current_stream() if stream is None else stream
+        self._fork.record(main)
+        self._side.wait_event(self._fork)
+        side = self._side
         b.gather_multi([x_t, v], self.edit_idx, self.n_edit, [self.x_e, self.v_e], dev_status=st,
-                       stream=stream)
+                       stream=side)
+        b.velocity_decay(self.v_e, scale, dt, self.x_e, self.n_edit, v_cache_out=self.v_avd,
+                         dev_status=st, stream=side)
+        b.merge(x_t, v, self.x_e, self.slot, dt_unedited, self.x_out, dev_status=st, stream=side)
+        self._join.record(side)
         b.rikv_store(k_full, v_full, self.cache_rows, self.n_cache, self.k_cache, self.v_cache,
                      dev_status=st, stream=stream)
         b.gather_multi([q_full, k_full, v_full], self.query_rows, self.n_q,
@@ -107,8 +124,6 @@ class RegionStep:
         if self.attention_events is not None:
             self.attention_events[1].record(stream)
         b.scatter(self.o_e, self.query_rows, self.n_q, self.o_full, dev_status=st, stream=stream)
-        b.velocity_decay(self.v_e, scale, dt, self.x_e, self.n_edit, v_cache_out=self.v_avd,
-                         dev_status=st, stream=stream)
-        b.merge(x_t, v, self.x_e, self.slot, dt_unedited, self.x_out, dev_status=st, stream=stream)
+        main.wait_event(self._join)
         self.launches += 10          # kernels launched (the attention call launches two)
         return self.x_out
