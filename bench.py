@@ -4,7 +4,7 @@
 A "step" is one pass of the whole hot path over one batch of synthetic input of
 the FLUX-Kontext-shaped workload (4096 image + 4096 reference + 512 text tokens,
 24 heads x 128, two-ellipse 20 % edit mask): partition, row lists, gathers, RIKV
-store, region attention, scatter, velocity decay + Euler, merge (9 library calls, 10 kernel launches).
+store, region attention, scatter, velocity decay + Euler, merge (8 library calls, 9 kernel launches).
 
 Prints ONE JSON line (rank 0).  `value` = region-attention FLOPs of the step
 divided by the whole step's device time (inputs resident in HBM).  `roofline`

@@ -88,6 +88,23 @@ int regione_partition(const regione_bf16* x_t, const regione_bf16* v, const regi
                       int32_t* n_edit, float* score, int32_t* dev_status, void* stream);
 
 /*
+ * regione_partition and regione_region_rows (below) in one launch: the partition
+ * of Sec. 4 "Adaptive Region Partition" that also writes the joint-sequence row
+ * lists of the region-attention layer (Sec. 4 "Region-Aware Generation").  Same
+ * arguments, layouts, limits and results as the two calls made one after the
+ * other; the row lists are composed while the index lists are written, so the
+ * second launch and its pass over the lists are saved.
+ */
+int regione_partition_rows(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
+                           int B, int N, int C, float t, int metric, float threshold,
+                           uint8_t* mask, int32_t* edit_idx, int32_t* keep_idx, int32_t* slot,
+                           int32_t* n_edit, float* score,
+                           int n_text, int n_ref, int membership,
+                           int32_t* query_rows, int32_t* n_query, int q_cap,
+                           int32_t* cache_rows, int32_t* n_cache, int c_cap,
+                           int32_t* dev_status, void* stream);
+
+/*
  * Morphological opening then closing of the edited mask on the rows x cols token
  * grid (Sec. 4, "Adaptive Region Partition": "morphological opening and closing
  * operations"; Algorithm 1 calls it Erosion_&_Dilate), followed by the same

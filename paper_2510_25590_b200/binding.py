@@ -26,6 +26,9 @@ SIGNATURES = {
     "regione_status_string": (c_char_p, [c_int]),
     "regione_partition": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_float, c_int, c_float,
                                   _P, _P, _P, _P, _P, _P, _P, _P]),
+    "regione_partition_rows": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_float, c_int, c_float,
+                                       _P, _P, _P, _P, _P, _P, c_int, c_int, c_int,
+                                       _P, _P, c_int, _P, _P, c_int, _P, _P]),
     "regione_mask_open_close": (c_int, [_P, c_int, c_int, c_int, _P, _P, _P, _P, _P, _P, _P]),
     "regione_region_rows": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_int, c_int,
                                     _P, _P, c_int, _P, _P, c_int, _P, _P]),
@@ -118,6 +121,23 @@ def partition(x_t, v, ref, t, metric, threshold, mask, edit_idx, keep_idx, slot,
         _ptr(keep_idx, torch.int32, "keep_idx"), _ptr(slot, torch.int32, "slot"),
         _ptr(n_edit, torch.int32, "n_edit"), _ptr(score, torch.float32, "score"),
         _ptr(dev_status, torch.int32, "dev_status"), _stream(stream)), "regione_partition")
+
+
+def partition_rows(x_t, v, ref, t, metric, threshold, mask, edit_idx, keep_idx, slot, n_edit,
+                   n_text, n_ref, membership, query_rows, n_query, cache_rows, n_cache,
+                   score=None, dev_status=None, stream=None):
+    """``partition`` and ``region_rows`` in one launch."""
+    torch = _torch()
+    B, N, C = x_t.shape
+    bf, i32 = torch.bfloat16, torch.int32
+    _check(load().regione_partition_rows(
+        _ptr(x_t, bf, "x_t"), _ptr(v, bf, "v"), _ptr(ref, bf, "ref"), B, N, C, float(t), int(metric),
+        float(threshold), _ptr(mask, torch.uint8, "mask"), _ptr(edit_idx, i32, "edit_idx"),
+        _ptr(keep_idx, i32, "keep_idx"), _ptr(slot, i32, "slot"), _ptr(n_edit, i32, "n_edit"),
+        _ptr(score, torch.float32, "score"), int(n_text), int(n_ref), int(membership),
+        _ptr(query_rows, i32), _ptr(n_query, i32), query_rows.shape[1],
+        _ptr(cache_rows, i32), _ptr(n_cache, i32), cache_rows.shape[1],
+        _ptr(dev_status, i32, "dev_status"), _stream(stream)), "regione_partition_rows")
 
 
 def mask_open_close(mask_in, rows, cols, mask_out, edit_idx, keep_idx, slot, n_edit,

@@ -60,11 +60,24 @@ __device__ int block_popc_scan(const uint32_t* bits, int* prefix, int nwords, in
     return carry;
 }
 
+// Optional second output of the partition: the joint-sequence row lists of one region-attention
+// layer (what regione_region_rows composes from the index lists), written in the same launch.
+struct RowLists {
+    int32_t* query_rows;     // nullptr: not requested
+    int32_t* n_query;
+    int32_t* cache_rows;
+    int32_t* n_cache;
+    int n_text, n_ref, membership, q_cap, c_cap;
+};
+
 // Writes mask / slot / edit_idx / keep_idx for tokens [start, start+ntok) of one request from
 // the mask words in shared memory.  edit_base / keep_base: entries preceding this CTA's share.
+// With row lists requested, an edited token n also becomes query row n_text + n and a kept token
+// cache row n_text + n, at the positions `q_off` / `c_off` further into this request's lists.
 __device__ void emit_indices(const uint32_t* bits, const int* prefix, int start, int ntok, int N,
                              int edit_base, int keep_base, uint8_t* mask, int32_t* edit_idx,
-                             int32_t* keep_idx, int32_t* slot) {
+                             int32_t* keep_idx, int32_t* slot, const RowLists& rl,
+                             int32_t* query_rows, int32_t* cache_rows, int q_off, int c_off) {
     for (int tl = threadIdx.x; tl < ntok; tl += blockDim.x) {
         const int n = start + tl;
         if (n >= N) break;
@@ -76,9 +89,13 @@ __device__ void emit_indices(const uint32_t* bits, const int* prefix, int start,
         if (edited) {
             slot[n] = edit_base + er;
             edit_idx[edit_base + er] = n;
+            if (query_rows != nullptr && q_off + edit_base + er < rl.q_cap)
+                query_rows[q_off + edit_base + er] = rl.n_text + n;
         } else {
             slot[n] = -1;
             keep_idx[keep_base + (tl - er)] = n;
+            if (cache_rows != nullptr && c_off + keep_base + (tl - er) < rl.c_cap)
+                cache_rows[c_off + keep_base + (tl - er)] = rl.n_text + n;
         }
     }
 }
@@ -112,7 +129,8 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
                  const uint16_t* __restrict__ ref, int N, int C, int share, float t, int metric,
                  float threshold, uint8_t* __restrict__ mask, int32_t* __restrict__ edit_idx,
                  int32_t* __restrict__ keep_idx, int32_t* __restrict__ slot,
-                 int32_t* __restrict__ n_edit, float* __restrict__ score) {
+                 int32_t* __restrict__ n_edit, float* __restrict__ score, const RowLists rl,
+                 int32_t* dev_status) {
     grid_dependency_wait();
     grid_launch_dependents();
     extern __shared__ uint32_t smem_u32[];
@@ -203,11 +221,38 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
     const int keep_base = start - edit_base;     // every token before `start` exists (start <= N)
 
     // ---- phase 3: coalesced per-token writes --------------------------------------------
+    const bool lists = rl.query_rows != nullptr;
+    const int q_text = (rl.membership == REGIONE_ROWS_PAPER) ? rl.n_text : 0;     // text rows are queries
+    const int c_text = (rl.membership == REGIONE_ROWS_PAPER) ? 0 : rl.n_text;     // ... or cached
+    int32_t* const q_rows = lists ? rl.query_rows + (size_t)b * rl.q_cap : nullptr;
+    int32_t* const c_rows = lists ? rl.cache_rows + (size_t)b * rl.c_cap : nullptr;
     if (start < N) {
         emit_indices(bits, prefix, start, share, N, edit_base, keep_base, mask + req,
-                     edit_idx + req, keep_idx + req, slot + req);
+                     edit_idx + req, keep_idx + req, slot + req, rl, q_rows, c_rows, q_text, c_text);
     }
     if (rank == csize - 1 && threadIdx.x == 0) n_edit[b] = edit_base + total;
+    if (lists) {
+        // rows that do not depend on the mask: the text rows and the reference rows, spread over
+        // the cluster's threads; the request's totals come from every rank's count
+        int ne_all = 0;
+        for (int r = 0; r < csize; ++r) ne_all += *cluster.map_shared_rank(&cta_count, r);
+        const int nu_all = N - ne_all;
+        const int stride = csize * blockDim.x;
+        for (int i = rank * blockDim.x + threadIdx.x; i < rl.n_text; i += stride) {
+            if (q_text > 0) { if (i < rl.q_cap) q_rows[i] = i; }
+            else if (i < rl.c_cap) c_rows[i] = i;
+        }
+        for (int i = rank * blockDim.x + threadIdx.x; i < rl.n_ref; i += stride) {
+            const int at = c_text + nu_all + i;
+            if (at < rl.c_cap) c_rows[at] = rl.n_text + N + i;
+        }
+        if (rank == csize - 1 && threadIdx.x == 0) {
+            const int nq = q_text + ne_all, nc = c_text + nu_all + rl.n_ref;
+            if (nq > rl.q_cap || nc > rl.c_cap) record_status(dev_status, REGIONE_DEV_BOUNDS);
+            rl.n_query[b] = min(nq, rl.q_cap);
+            rl.n_cache[b] = min(nc, rl.c_cap);
+        }
+    }
     cluster.sync();                              // peers may still be reading cta_count
 }
 
@@ -263,8 +308,9 @@ mask_open_close_kernel(const uint8_t* __restrict__ mask_in, int rows, int cols,
     }
     __syncthreads();
     const int total = block_popc_scan(bits, prefix, nwords, warp_tot);
+    const RowLists none = {};
     emit_indices(bits, prefix, 0, nwords * 32, N, 0, 0, mask_out + req, edit_idx + req,
-                 keep_idx + req, slot + req);
+                 keep_idx + req, slot + req, none, nullptr, nullptr, 0, 0);
     if (threadIdx.x == 0) n_edit[b] = total;
 }
 
@@ -317,7 +363,8 @@ static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st
                                     const uint16_t* x_t, const uint16_t* v, const uint16_t* ref,
                                     int N, int C, float t, int metric, float thr, uint8_t* mask,
                                     int32_t* edit_idx, int32_t* keep_idx, int32_t* slot,
-                                    int32_t* n_edit, float* score) {
+                                    int32_t* n_edit, float* score, const RowLists& rl,
+                                    int32_t* dev_status) {
     cudaLaunchConfig_t cfg = {};
     // enough warps per CTA to keep the loads of a large share in flight (a cluster is at most 8
     // CTAs, so a long request cannot get its memory parallelism from the grid); 512 threads let
@@ -337,15 +384,13 @@ static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, partition_kernel<L>, x_t, v, ref, N, C, share, t, metric, thr,
-                              mask, edit_idx, keep_idx, slot, n_edit, score);
+                              mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status);
 }
 
-extern "C" int regione_partition(const regione_bf16* x_t, const regione_bf16* v,
-                                 const regione_bf16* ref, int B, int N, int C, float t, int metric,
-                                 float threshold, uint8_t* mask, int32_t* edit_idx,
-                                 int32_t* keep_idx, int32_t* slot, int32_t* n_edit, float* score,
-                                 int32_t* dev_status, void* stream) {
-    (void)dev_status;
+static int partition_impl(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
+                          int B, int N, int C, float t, int metric, float threshold, uint8_t* mask,
+                          int32_t* edit_idx, int32_t* keep_idx, int32_t* slot, int32_t* n_edit,
+                          float* score, const RowLists& rl, int32_t* dev_status, void* stream) {
     if (!x_t || !v || !ref || !mask || !edit_idx || !keep_idx || !slot || !n_edit)
         return REGIONE_INVALID_ARG;
     if (B < 0 || N < 1 || C < 1) return REGIONE_INVALID_ARG;
@@ -365,7 +410,7 @@ extern "C" int regione_partition(const regione_bf16* x_t, const regione_bf16* v,
 #define REGIONE_PART_CASE(LL)                                                                   \
     case LL:                                                                                    \
         e = launch_partition<LL>(csize, B, share, st, x_t, v, ref, N, C, t, metric, threshold,  \
-                                 mask, edit_idx, keep_idx, slot, n_edit, score);                \
+                                 mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status); \
         break;
     switch (L) {
         REGIONE_PART_CASE(1)
@@ -375,10 +420,38 @@ extern "C" int regione_partition(const regione_bf16* x_t, const regione_bf16* v,
         REGIONE_PART_CASE(16)
         default:
             e = launch_partition<32>(csize, B, share, st, x_t, v, ref, N, C, t, metric, threshold,
-                                     mask, edit_idx, keep_idx, slot, n_edit, score);
+                                     mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status);
     }
 #undef REGIONE_PART_CASE
     return launch_status(e);
+}
+
+extern "C" int regione_partition(const regione_bf16* x_t, const regione_bf16* v,
+                                 const regione_bf16* ref, int B, int N, int C, float t, int metric,
+                                 float threshold, uint8_t* mask, int32_t* edit_idx,
+                                 int32_t* keep_idx, int32_t* slot, int32_t* n_edit, float* score,
+                                 int32_t* dev_status, void* stream) {
+    RowLists none = {};
+    return partition_impl(x_t, v, ref, B, N, C, t, metric, threshold, mask, edit_idx, keep_idx, slot,
+                          n_edit, score, none, dev_status, stream);
+}
+
+extern "C" int regione_partition_rows(const regione_bf16* x_t, const regione_bf16* v,
+                                      const regione_bf16* ref, int B, int N, int C, float t,
+                                      int metric, float threshold, uint8_t* mask, int32_t* edit_idx,
+                                      int32_t* keep_idx, int32_t* slot, int32_t* n_edit, float* score,
+                                      int n_text, int n_ref, int membership, int32_t* query_rows,
+                                      int32_t* n_query, int q_cap, int32_t* cache_rows,
+                                      int32_t* n_cache, int c_cap, int32_t* dev_status, void* stream) {
+    if (!query_rows || !n_query || !cache_rows || !n_cache) return REGIONE_INVALID_ARG;
+    if (n_text < 0 || n_ref < 0 || q_cap < 0 || c_cap < 0) return REGIONE_INVALID_ARG;
+    if (membership != REGIONE_ROWS_EDITED_QUERIES && membership != REGIONE_ROWS_PAPER)
+        return REGIONE_INVALID_ARG;
+    RowLists rl;
+    rl.query_rows = query_rows; rl.n_query = n_query; rl.cache_rows = cache_rows; rl.n_cache = n_cache;
+    rl.n_text = n_text; rl.n_ref = n_ref; rl.membership = membership; rl.q_cap = q_cap; rl.c_cap = c_cap;
+    return partition_impl(x_t, v, ref, B, N, C, t, metric, threshold, mask, edit_idx, keep_idx, slot,
+                          n_edit, score, rl, dev_status, stream);
 }
 
 extern "C" int regione_mask_open_close(const uint8_t* mask_in, int B, int rows, int cols,

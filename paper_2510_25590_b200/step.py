@@ -4,7 +4,8 @@ This is call sequencing and buffer ownership only (torch tensors are device
 buffers): every operation runs in the library's kernels.  The sequence follows
 Algorithm 1 of the paper for one layer:
 
-  partition -> row lists -> two independent branches, joined before the step returns:
+  partition with the joint-sequence row lists (one launch) -> two independent branches, joined
+  before the step returns:
     attention branch: RIKV store -> gather Q/K/V of the recomputed rows (one launch) ->
                       region attention -> scatter the attention rows back
     latent branch   : gather X^E, v^E (one launch) -> velocity decay + Euler update -> merge with
@@ -93,11 +94,10 @@ class RegionStep:
         s = self.shp
         st = self.dev_status
         b = binding
-        b.partition(x_t, v, ref, t, s.metric, s.threshold, self.mask, self.edit_idx, self.keep_idx,
-                    self.slot, self.n_edit, dev_status=st, stream=stream)
-        b.region_rows(self.edit_idx, self.keep_idx, self.n_edit, s.n_text, s.n_ref, s.membership,
-                      self.query_rows, self.n_q, self.cache_rows, self.n_cache, dev_status=st,
-                      stream=stream)
+        b.partition_rows(x_t, v, ref, t, s.metric, s.threshold, self.mask, self.edit_idx,
+                         self.keep_idx, self.slot, self.n_edit, s.n_text, s.n_ref, s.membership,
+                         self.query_rows, self.n_q, self.cache_rows, self.n_cache, dev_status=st,
+                         stream=stream)
         # Two independent branches hang off the partition: the latent branch (gather of X^E and v,
         # velocity decay, merge: small latency-bound kernels) and the attention branch (cache store,
         # gather of Q/K/V, attention, scatter).  The latent branch runs on a side stream so that it
@@ -125,5 +125,5 @@ class RegionStep:
             self.attention_events[1].record(stream)
         b.scatter(self.o_e, self.query_rows, self.n_q, self.o_full, dev_status=st, stream=stream)
         main.wait_event(self._join)
-        self.launches += 10          # kernels launched (the attention call launches two)
+        self.launches += 9           # kernels launched (the attention call launches two)
         return self.x_out

@@ -168,3 +168,61 @@ def test_region_rows_match_generator_layout(membership):
         assert np.array_equal(qr[b, :int(nq[b])].cpu().numpy(), want["query"])
         assert np.array_equal(cr[b, :int(nc[b])].cpu().numpy(), want["cache"])
         assert np.all(qr[b, int(nq[b]):].cpu().numpy() == -7)
+
+
+@pytest.mark.parametrize("membership", ["edited_queries", "paper"])
+@pytest.mark.parametrize("grid,n_text,batch", [((48, 48), 77, 3), ((64, 64), 512, 1), ((9, 7), 0, 2), ((96, 96), 33, 2)])
+def test_partition_with_row_lists_in_one_launch(membership, grid, n_text, batch):
+    """regione_partition_rows = regione_partition + regione_region_rows: every output bit-exact
+    against the oracle partition and the generator's row layout, tails untouched."""
+    import torch
+    wl = synth.scaled_workload(synth.WORKLOADS[5], grid=grid, n_text=n_text, batch=batch)
+    lat = synth.make_latents(wl)
+    p = orc.partition(lat["x_t"], lat["v"], lat["ref"], lat["t"], orc.COSINE, wl.threshold)
+    B, N = wl.batch, wl.n_img
+    q_cap, c_cap = N + wl.n_text + 3, wl.n_full + 5
+    i32 = torch.int32
+    mask = torch.full((B, N), 77, dtype=torch.uint8, device="cuda")
+    e, k, s = (torch.full((B, N), -7, dtype=i32, device="cuda") for _ in range(3))
+    ne = torch.full((B,), -7, dtype=i32, device="cuda")
+    qr = torch.full((B, q_cap), -7, dtype=i32, device="cuda")
+    cr = torch.full((B, c_cap), -7, dtype=i32, device="cuda")
+    nq, nc = (torch.full((B,), -7, dtype=i32, device="cuda") for _ in range(2))
+    st = torch.zeros(1, dtype=i32, device="cuda")
+    score = torch.full((B, N), float("nan"), dtype=torch.float32, device="cuda")
+    binding.partition_rows(dev_bf16(lat["x_t"]), dev_bf16(lat["v"]), dev_bf16(lat["ref"]), lat["t"],
+                           binding.METRIC_COSINE, wl.threshold, mask, e, k, s, ne, wl.n_text, wl.n_ref,
+                           binding.ROWS_PAPER if membership == "paper" else binding.ROWS_EDITED_QUERIES,
+                           qr, nq, cr, nc, score=score, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st[0]) == 0
+    got = dict(mask=mask.cpu().numpy(), edit_idx=e.cpu().numpy(), keep_idx=k.cpu().numpy(),
+               slot=s.cpu().numpy(), n_edit=ne.cpu().numpy(), score=score.cpu().numpy())
+    check_against_oracle(got, p, N)
+    for b in range(B):
+        want = synth.region_rows(wl, p["mask"][b], membership)
+        assert int(nq[b]) == len(want["query"]) and int(nc[b]) == len(want["cache"])
+        assert np.array_equal(qr[b, :int(nq[b])].cpu().numpy(), want["query"])
+        assert np.array_equal(cr[b, :int(nc[b])].cpu().numpy(), want["cache"])
+        assert np.all(qr[b, int(nq[b]):].cpu().numpy() == -7)
+        assert np.all(cr[b, int(nc[b]):].cpu().numpy() == -7)
+
+
+def test_partition_with_row_lists_reports_lists_that_do_not_fit():
+    import torch
+    wl = synth.scaled_workload(synth.WORKLOADS[5], grid=(32, 32), n_text=16, batch=1)
+    lat = synth.make_latents(wl)
+    B, N = wl.batch, wl.n_img
+    i32 = torch.int32
+    mask = torch.zeros((B, N), dtype=torch.uint8, device="cuda")
+    e, k, s = (torch.zeros((B, N), dtype=i32, device="cuda") for _ in range(3))
+    ne, nq, nc = (torch.zeros(B, dtype=i32, device="cuda") for _ in range(3))
+    qr = torch.full((B, 8), -7, dtype=i32, device="cuda")            # far too small
+    cr = torch.full((B, 8), -7, dtype=i32, device="cuda")
+    st = torch.zeros(1, dtype=i32, device="cuda")
+    binding.partition_rows(dev_bf16(lat["x_t"]), dev_bf16(lat["v"]), dev_bf16(lat["ref"]), lat["t"],
+                           binding.METRIC_COSINE, wl.threshold, mask, e, k, s, ne, wl.n_text, wl.n_ref,
+                           binding.ROWS_EDITED_QUERIES, qr, nq, cr, nc, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st[0]) == binding.DEV_BOUNDS
+    assert int(nq[0]) == 8 and int(nc[0]) == 8                       # clamped, nothing written past the end

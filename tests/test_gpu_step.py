@@ -69,7 +69,7 @@ def test_zero_edit_mask_is_one_step_prediction_everywhere():
 
 
 def test_step_replayed_from_a_cuda_graph_matches_the_eager_step():
-    """The ten launches of a step (each with programmatic stream serialization) captured into a
+    """The launches of a step (each with programmatic stream serialization, two streams) captured into a
     CUDA graph and replayed give bit-identical buffers to the same step launched eagerly."""
     import torch
     wl = synth.scaled_workload(synth.WORKLOADS[2], grid=(24, 24), n_text=70)
