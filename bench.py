@@ -4,7 +4,8 @@
 A "step" is one pass of the whole hot path over one batch of synthetic input of
 the FLUX-Kontext-shaped workload (4096 image + 4096 reference + 512 text tokens,
 24 heads x 128, two-ellipse 20 % edit mask): partition, row lists, gathers, RIKV
-store, region attention, scatter, velocity decay + Euler, merge (8 library calls, 9 kernel launches).
+store, region attention with its rows scattered back, velocity decay + Euler, merge (7 library calls,
+8 kernel launches on two streams).
 
 Prints ONE JSON line (rank 0).  `value` = region-attention FLOPs of the step
 divided by the whole step's device time (inputs resident in HBM).  `roofline`
@@ -424,6 +425,8 @@ def run_ours(args):
         for k in host:
             d[k].copy_(host[k], non_blocking=True)
         one()
+        # the step leaves the attention rows at their joint-sequence positions; the host wants them dense
+        binding.gather(step.o_full, step.query_rows, step.n_q, step.o_e, dev_status=step.dev_status)
         out_host.copy_(step.x_out, non_blocking=True)
         o_host.copy_(step.o_e, non_blocking=True)
 

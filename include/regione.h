@@ -220,6 +220,28 @@ int regione_region_attention(const regione_bf16* q,
                              int32_t* dev_status, void* stream);
 
 /*
+ * regione_region_attention followed by regione_scatter of its rows, in the same
+ * launches (Sec. 4: the attention rows of the recomputed tokens are put back at
+ * their positions in the joint sequence): the result of query row i of request b
+ * is written to out_full[b, out_rows[b, i], :, :] instead of out[b, i, :, :].
+ *
+ * out_full : dev bf16 [B, out_rows_cap, H, D]; rows not named by out_rows[b, 0..n_q[b])
+ *            are left untouched
+ * out_rows : dev int32 [B, Nq_cap]; an entry outside [0, out_rows_cap) drops that
+ *            row and records REGIONE_DEV_BOUNDS
+ * Everything else as regione_region_attention (same workspace query).
+ */
+int regione_region_attention_scatter(const regione_bf16* q,
+                                     const regione_bf16* k_fresh, const regione_bf16* v_fresh,
+                                     const regione_bf16* k_cache, const regione_bf16* v_cache,
+                                     const int32_t* n_q, const int32_t* n_fresh, const int32_t* n_cache,
+                                     int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D,
+                                     float softmax_scale, regione_bf16* out_full, int out_rows_cap,
+                                     const int32_t* out_rows,
+                                     void* workspace, size_t workspace_bytes,
+                                     int32_t* dev_status, void* stream);
+
+/*
  * Region attention that brings its own scratch memory.  (The paper has no
  * counterpart: this entry point exists only for the way the library is deployed.)
  *

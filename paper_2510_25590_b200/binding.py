@@ -38,6 +38,7 @@ SIGNATURES = {
     "regione_rikv_store": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
     "regione_region_attention_workspace": (c_size_t, [c_int] * 6),
     "regione_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, c_size_t, _P, _P]),
+    "regione_region_attention_scatter": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, c_int, _P, _P, c_size_t, _P, _P]),
     "regione_region_attention_static": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, _P]),
     "regione_avd_step": (c_int, [POINTER(c_double), c_double, c_double, c_double, POINTER(c_int)]),
     "regione_gamma_fit": (c_int, [_P, c_int, c_int, c_int64, _P, _P, _P, _P]),
@@ -237,6 +238,27 @@ def region_attention(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cach
         _ptr(n_cache, i32), B, Nq_cap, Nf_cap, Nc_cap, H, D, float(softmax_scale), _ptr(out, bf, "out"),
         _ptr(workspace, None, "workspace"), ws_bytes, _ptr(dev_status, i32), _stream(stream)),
         "regione_region_attention")
+
+
+def region_attention_scatter(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, out_full,
+                             out_rows, softmax_scale=0.0, workspace=None, dev_status=None, stream=None):
+    """``region_attention`` whose row i of request b lands in out_full[b, out_rows[b, i]]."""
+    torch = _torch()
+    bf = torch.bfloat16
+    B, Nq_cap, H, D = q.shape
+    Nf_cap = 0 if k_fresh is None else k_fresh.shape[1]
+    Nc_cap = 0 if k_cache is None else k_cache.shape[1]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    i32 = torch.int32
+    if out_rows.shape[0] != B or out_rows.shape[1] != Nq_cap:
+        raise RegionEError("out_rows must be [B, Nq_cap]")
+    _check(load().regione_region_attention_scatter(
+        _ptr(q, bf, "q"), _ptr(k_fresh, bf, "k_fresh"), _ptr(v_fresh, bf, "v_fresh"),
+        _ptr(k_cache, bf, "k_cache"), _ptr(v_cache, bf, "v_cache"), _ptr(n_q, i32), _ptr(n_fresh, i32),
+        _ptr(n_cache, i32), B, Nq_cap, Nf_cap, Nc_cap, H, D, float(softmax_scale),
+        _ptr(out_full, bf, "out_full"), out_full.shape[1], _ptr(out_rows, i32, "out_rows"),
+        _ptr(workspace, None, "workspace"), ws_bytes, _ptr(dev_status, i32), _stream(stream)),
+        "regione_region_attention_scatter")
 
 
 def region_attention_static(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, out,

@@ -14,8 +14,8 @@ int launch_region_attention_simt(const uint16_t*, const uint16_t*, const uint16_
 size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D);
 int launch_region_attention_tc(const uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*,
                                const uint16_t*, const int32_t*, const int32_t*, const int32_t*, int,
-                               int, int, int, int, int, float, uint16_t*, void*, size_t, int32_t*,
-                               cudaStream_t);
+                               int, int, int, int, int, float, uint16_t*, const int32_t*, int, void*,
+                               size_t, int32_t*, cudaStream_t);
 }  // namespace regione
 
 using namespace regione;
@@ -60,13 +60,15 @@ extern "C" size_t regione_region_attention_workspace(int B, int Nq_cap, int Nf_c
     return region_attention_tc_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D);
 }
 
-extern "C" int regione_region_attention(const regione_bf16* q, const regione_bf16* k_fresh,
-                                        const regione_bf16* v_fresh, const regione_bf16* k_cache,
-                                        const regione_bf16* v_cache, const int32_t* n_q,
-                                        const int32_t* n_fresh, const int32_t* n_cache, int B,
-                                        int Nq_cap, int Nf_cap, int Nc_cap, int H, int D,
-                                        float softmax_scale, regione_bf16* out, void* workspace,
-                                        size_t workspace_bytes, int32_t* dev_status, void* stream) {
+// Shared body of regione_region_attention (out_rows == nullptr) and regione_region_attention_scatter.
+static int region_attention_impl(const regione_bf16* q, const regione_bf16* k_fresh,
+                                 const regione_bf16* v_fresh, const regione_bf16* k_cache,
+                                 const regione_bf16* v_cache, const int32_t* n_q,
+                                 const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap,
+                                 int Nf_cap, int Nc_cap, int H, int D, float softmax_scale,
+                                 regione_bf16* out, const int32_t* out_rows, int out_cap,
+                                 void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                 void* stream) {
     if (!q || !out || !n_q || !n_fresh || !n_cache) return REGIONE_INVALID_ARG;
     if (B < 0 || Nq_cap < 0 || Nf_cap < 0 || Nc_cap < 0 || H < 1) return REGIONE_INVALID_ARG;
     if (Nf_cap > 0 && (!k_fresh || !v_fresh)) return REGIONE_INVALID_ARG;
@@ -79,16 +81,42 @@ extern "C" int regione_region_attention(const regione_bf16* q, const regione_bf1
     if (B == 0 || Nq_cap == 0) return REGIONE_OK;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = (cudaStream_t)stream;
-    if (use_simt())
+    if (use_simt()) {
+        if (out_rows != nullptr) return REGIONE_UNSUPPORTED;   // the cross-check path writes dense rows
         return launch_region_attention_simt(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh,
                                             n_cache, B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out,
                                             dev_status, st);
+    }
     const size_t need = region_attention_tc_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D);
     if (need > 0) {
         if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return REGIONE_INVALID_ARG;
         if (workspace_bytes < need) return REGIONE_WORKSPACE_TOO_SMALL;
     }
     return launch_region_attention_tc(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
-                                      B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, workspace,
-                                      workspace_bytes, dev_status, st);
+                                      B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, out_rows, out_cap,
+                                      workspace, workspace_bytes, dev_status, st);
+}
+
+extern "C" int regione_region_attention(const regione_bf16* q, const regione_bf16* k_fresh,
+                                        const regione_bf16* v_fresh, const regione_bf16* k_cache,
+                                        const regione_bf16* v_cache, const int32_t* n_q,
+                                        const int32_t* n_fresh, const int32_t* n_cache, int B,
+                                        int Nq_cap, int Nf_cap, int Nc_cap, int H, int D,
+                                        float softmax_scale, regione_bf16* out, void* workspace,
+                                        size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    return region_attention_impl(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, B,
+                                 Nq_cap, Nf_cap, Nc_cap, H, D, softmax_scale, out, nullptr, 0,
+                                 workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" int regione_region_attention_scatter(
+    const regione_bf16* q, const regione_bf16* k_fresh, const regione_bf16* v_fresh,
+    const regione_bf16* k_cache, const regione_bf16* v_cache, const int32_t* n_q,
+    const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap, int Nf_cap, int Nc_cap, int H,
+    int D, float softmax_scale, regione_bf16* out_full, int out_rows_cap, const int32_t* out_rows,
+    void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    if (!out_rows || out_rows_cap < 1) return REGIONE_INVALID_ARG;
+    return region_attention_impl(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, B,
+                                 Nq_cap, Nf_cap, Nc_cap, H, D, softmax_scale, out_full, out_rows,
+                                 out_rows_cap, workspace, workspace_bytes, dev_status, stream);
 }

@@ -114,7 +114,9 @@ struct AttnParams {
     int P_cap;           // query pairs per (request, head) at capacity
     int max_slots;       // workspace slots per item (>= 2)
     float scale_log2e;
-    uint16_t* out;
+    uint16_t* out;       // [B, out_cap, H, D]
+    const int32_t* out_rows;   // nullptr: query row i goes to out row i; else to row out_rows[b, i]
+    int out_cap;         // rows per request of `out` (Nq_cap without out_rows)
     int32_t* dev_status;
     float* part_o;       // [B, H, P_cap, max_slots, 256, D] unnormalised outputs
     float2* part_ml;     // [B, H, P_cap, max_slots, 256]    (running max in the exp2 domain, sum)
@@ -574,6 +576,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
+
         const int n_my = n_tiles > 0 ? role_tiles(t) : 0;
         for (int j = 0; j < n_my; ++j) {
             bool cached; int row0, valid;
@@ -669,6 +672,11 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         const int wrow0 = q0 + (split ? 0 : t) * kBM + ((warp & 3) << 5);   // first query row of this warp
         const int live_rows = min(max(nq - wrow0, 0), 32);
         const bool live = lane < live_rows;
+        // where this thread's query row goes in `out` (-1: the row is dead); the lookup is issued
+        // ahead of the wait for the last product and used after it
+        int dst_row = -1;
+        if (live && direct)
+            dst_row = p.out_rows != nullptr ? p.out_rows[(size_t)b * p.Nq_cap + wrow0 + lane] : wrow0 + lane;
         if (n_tiles > 0 && ok) {
             ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status);
             if (ok) ptx::tc_fence_after_sync();
@@ -706,7 +714,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         };
         if (!(split && t == 1)) {
         uint8_t* const stage = smem_gen + t * kTileBytes + (warp & 3) * (kTileBytes / 4);
-        auto store_pieces = [&](const uint4 (&v)[8], uint8_t* g_row0, size_t row_stride) {
+        // `to` = this lane's destination row (counted from g_row0), -1 to drop the row
+        auto store_pieces = [&](const uint4 (&v)[8], uint8_t* g_row0, size_t row_stride, int to) {
             // piece q of row r sits at 16-byte column q ^ (r & 7): both the row-wise writes and
             // the piece-wise reads are free of bank conflicts without padding
             uint4* dst = reinterpret_cast<uint4*>(stage + lane * 128);
@@ -718,20 +727,25 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 const int rr = i * 4 + (lane >> 3);
                 const uint4 x = *reinterpret_cast<const uint4*>(stage + rr * 128 +
                                                                  (((lane & 7) ^ (rr & 7)) << 4));
-                if (rr < live_rows)
-                    *reinterpret_cast<uint4*>(g_row0 + rr * row_stride + (lane & 7) * 16) = x;
+                const int to_rr = __shfl_sync(0xffffffffu, to, rr);
+                if (to_rr >= 0)
+                    *reinterpret_cast<uint4*>(g_row0 + to_rr * row_stride + (lane & 7) * 16) = x;
             }
             __syncwarp();
         };
         if (direct) {
             // O / l -> bf16 -> out
+            if (dst_row >= p.out_cap || (dst_row < 0 && live)) {     // destination out of range: dropped
+                record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+                dst_row = -1;
+            }
             const size_t row_stride = (size_t)p.H * D * 2;
             uint8_t* g_row0 = reinterpret_cast<uint8_t*>(p.out) +
-                              (((size_t)b * p.Nq_cap + wrow0) * p.H + h) * D * 2;
+                              (((size_t)b * p.out_cap) * p.H + h) * D * 2;      // row 0 of the request
             if (n_tiles == 0) {
-                if (live)
+                if (dst_row >= 0)
                     for (int q = 0; q < D / 8; ++q)
-                        reinterpret_cast<uint4*>(g_row0 + lane * row_stride)[q] = make_uint4(0, 0, 0, 0);
+                        reinterpret_cast<uint4*>(g_row0 + dst_row * row_stride)[q] = make_uint4(0, 0, 0, 0);
             } else if (ok) {
                 const float inv = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll 1
@@ -753,7 +767,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                         v[q].z = pack_bf16x2(__uint_as_float(r[8 * q + 4]) * inv, __uint_as_float(r[8 * q + 5]) * inv);
                         v[q].w = pack_bf16x2(__uint_as_float(r[8 * q + 6]) * inv, __uint_as_float(r[8 * q + 7]) * inv);
                     }
-                    store_pieces(v, g_row0 + c64 * 128, row_stride);
+                    store_pieces(v, g_row0 + c64 * 128, row_stride, dst_row);
                 }
             }
         } else {
@@ -777,7 +791,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                     uint4 v[8];
 #pragma unroll
                     for (int q = 0; q < 8; ++q) v[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-                    store_pieces(v, g_row0 + ch * 128, (size_t)D * 4);
+                    store_pieces(v, g_row0 + ch * 128, (size_t)D * 4, live ? lane : -1);
                 }
                 if (live) p.part_ml[prow_w + lane] = make_float2(m, l);
             }
@@ -890,6 +904,8 @@ region_attention_combine_kernel(const AttnParams p) {
     if (qrow >= nq) return;
     const size_t item_idx = ((size_t)b * p.H + h) * p.P_cap + qp;
     const size_t prow0 = item_idx * p.max_slots * (2 * kBM) + r_local;
+    // (issued together with the slots' loads, used after them)
+    const int dst_row = p.out_rows != nullptr ? p.out_rows[(size_t)b * p.Nq_cap + qrow] : qrow;
 
     float2 ml[kCombineMaxSlots];
     Vec o[kCombineMaxSlots];
@@ -920,7 +936,11 @@ region_attention_combine_kernel(const AttnParams p) {
         }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
-    uint16_t* orow = p.out + (((size_t)b * p.Nq_cap + qrow) * p.H + h) * D + lane * E;
+    if (dst_row < 0 || dst_row >= p.out_cap) {             // destination out of range: dropped
+        if (lane == 0) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+        return;
+    }
+    uint16_t* orow = p.out + (((size_t)b * p.out_cap + dst_row) * p.H + h) * D + lane * E;
     uint32_t packed[E / 2];
 #pragma unroll
     for (int e = 0; e < E; e += 2) packed[e / 2] = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
@@ -1043,8 +1063,8 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
                                const uint16_t* k_cache, const uint16_t* v_cache, const int32_t* n_q,
                                const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap,
                                int Nf_cap, int Nc_cap, int H, int D, float scale, uint16_t* out,
-                               void* workspace, size_t workspace_bytes, int32_t* dev_status,
-                               cudaStream_t st) {
+                               const int32_t* out_rows, int out_cap, void* workspace,
+                               size_t workspace_bytes, int32_t* dev_status, cudaStream_t st) {
     (void)workspace_bytes;
     CUtensorMap maps[5];
     // an absent segment still needs a valid (never dereferenced) base address
@@ -1063,6 +1083,8 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
     prm.P_cap = lp.P_cap; prm.max_slots = lp.max_slots;
     prm.scale_log2e = scale * 1.4426950408889634f;
     prm.out = out; prm.dev_status = dev_status;
+    prm.out_rows = out_rows;
+    prm.out_cap = out_rows != nullptr ? out_cap : Nq_cap;
     const size_t rows = slot_rows(lp, B, H);
     prm.part_o = reinterpret_cast<float*>(workspace);
     uint8_t* const ws = reinterpret_cast<uint8_t*>(workspace);
@@ -1129,6 +1151,6 @@ extern "C" int regione_region_attention_static(
     // Nothing in the scratch has to start at zero: every word the merge kernel reads is written
     // by the attention kernel of the same call, so the previous call's contents are harmless.
     return launch_region_attention_tc(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
-                                      B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, scratch,
+                                      B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, nullptr, 0, scratch,
                                       kStaticScratchBytes, dev_status, (cudaStream_t)stream);
 }

@@ -7,7 +7,7 @@ Algorithm 1 of the paper for one layer:
   partition with the joint-sequence row lists (one launch) -> two independent branches, joined
   before the step returns:
     attention branch: RIKV store -> gather Q/K/V of the recomputed rows (one launch) ->
-                      region attention -> scatter the attention rows back
+                      region attention writing its rows back at their joint-sequence positions
     latent branch   : gather X^E, v^E (one launch) -> velocity decay + Euler update -> merge with
                       the one-step-predicted unedited tokens (on a side stream)
 
@@ -118,12 +118,12 @@ class RegionStep:
                        [self.q_e, self.k_fresh, self.v_fresh], dev_status=st, stream=stream)
         if self.attention_events is not None:
             self.attention_events[0].record(stream)
-        b.region_attention(self.q_e, self.k_fresh, self.v_fresh, self.k_cache, self.v_cache, self.n_q,
-                           self.n_q, self.n_cache, self.o_e, workspace=self.workspace, dev_status=st,
-                           stream=stream)
+        # the attention rows go straight to their positions in the joint sequence (o_full)
+        b.region_attention_scatter(self.q_e, self.k_fresh, self.v_fresh, self.k_cache, self.v_cache,
+                                   self.n_q, self.n_q, self.n_cache, self.o_full, self.query_rows,
+                                   workspace=self.workspace, dev_status=st, stream=stream)
         if self.attention_events is not None:
             self.attention_events[1].record(stream)
-        b.scatter(self.o_e, self.query_rows, self.n_q, self.o_full, dev_status=st, stream=stream)
         main.wait_event(self._join)
-        self.launches += 9           # kernels launched (the attention call launches two)
+        self.launches += 8           # kernels launched (the attention call launches two)
         return self.x_out

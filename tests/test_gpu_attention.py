@@ -279,3 +279,43 @@ def test_scheduling_plans(caps, counts):
             assert np.all(got[b, r, h] == 0.0)              # no key at all: the row is zero
     for b in range(B):
         assert np.all(got[b, n_q[b]:] == -3.0)              # rows past n_q are not written
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("counts", [[(300, 300, 2000)], [(100, 100, 647), (257, 200, 300)], [(5, 0, 0)]])
+def test_attention_with_scattered_output_rows(counts, D):
+    """regione_region_attention_scatter = regione_region_attention, then regione_scatter: the same
+    bits at the rows named by out_rows, every other row of the destination untouched."""
+    import torch
+    B, H = len(counts), 3
+    cap_q = max(c[0] for c in counts) + 2
+    cap_f = max(max(c[1] for c in counts), 1)
+    cap_c = max(max(c[2] for c in counts), 1)
+    n_full = cap_q + 300
+    rng = np.random.default_rng(17 + D + cap_q)
+    q = dev_bf16(_rand_bf16(rng, (B, cap_q, H, D), 0.5))
+    kf, vf = dev_bf16(_rand_bf16(rng, (B, cap_f, H, D), 0.5)), dev_bf16(_rand_bf16(rng, (B, cap_f, H, D)))
+    kc, vc = dev_bf16(_rand_bf16(rng, (B, cap_c, H, D), 0.5)), dev_bf16(_rand_bf16(rng, (B, cap_c, H, D)))
+    n_q, n_f, n_c = (dev_i32(np.array([c[i] for c in counts], np.int32)) for i in range(3))
+    rows = np.stack([np.sort(rng.permutation(n_full)[:cap_q]) for _ in range(B)]).astype(np.int32)
+    d_rows = dev_i32(rows)
+    ws = torch.empty(max(binding.region_attention_workspace(B, cap_q, cap_f, cap_c, H, D), 256),
+                     dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dense = torch.full((B, cap_q, H, D), -3.0, dtype=torch.bfloat16, device="cuda")
+    binding.region_attention(q, kf, vf, kc, vc, n_q, n_f, n_c, dense, workspace=ws, dev_status=st)
+    want = torch.full((B, n_full, H, D), -5.0, dtype=torch.bfloat16, device="cuda")
+    binding.scatter(dense, d_rows, n_q, want, dev_status=st)
+    got = torch.full((B, n_full, H, D), -5.0, dtype=torch.bfloat16, device="cuda")
+    binding.region_attention_scatter(q, kf, vf, kc, vc, n_q, n_f, n_c, got, d_rows, workspace=ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st[0]) == 0
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    # a destination outside the tensor is dropped and reported; the other rows still arrive
+    bad = rows.copy(); bad[0, 0] = n_full + 7
+    got2 = torch.full((B, n_full, H, D), -5.0, dtype=torch.bfloat16, device="cuda")
+    binding.region_attention_scatter(q, kf, vf, kc, vc, n_q, n_f, n_c, got2, dev_i32(bad), workspace=ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st[0]) == binding.DEV_BOUNDS
+    want[0, rows[0, 0]] = -5.0
+    assert torch.equal(got2.view(torch.int16), want.view(torch.int16))

@@ -41,7 +41,8 @@ def run_step(wl, membership="edited_queries", ratio=None):
         assert np.array_equal(step.cache_rows[b, :nc].cpu().numpy(), want["cache_rows"][b, :nc])
         assert np.array_equal(host_f64(step.k_cache[b, :nc]), want["k_cache"][b, :nc])      # copies: bit-exact
         assert np.array_equal(host_f64(step.v_cache[b, :nc]), want["v_cache"][b, :nc])
-        assert_close(host_f64(step.o_e[b, :nq]), want["o_e"][b, :nq], "attention rows")
+        o_rows = step.o_full[b][step.query_rows[b, :nq].long()]      # attention rows, where the step put them
+        assert_close(host_f64(o_rows), want["o_e"][b, :nq], "attention rows")
         ne = int(p["n_edit"][b])
         assert_close(host_f64(step.x_e[b, :ne]), want["x_e"][b, :ne], "x_e")
     assert_close(host_f64(step.o_full), want["o_full"], "scattered attention output")
@@ -82,7 +83,7 @@ def test_step_replayed_from_a_cuda_graph_matches_the_eager_step():
     shp = StepShapes(wl.batch, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads, wl.head_dim, cap,
                      binding.METRIC_COSINE, wl.threshold, binding.ROWS_EDITED_QUERIES)
     step = RegionStep(shp)
-    names = ("mask", "slot", "n_edit", "k_cache", "v_cache", "o_e", "o_full", "x_e", "x_out")
+    names = ("mask", "slot", "n_edit", "k_cache", "v_cache", "o_full", "x_e", "x_out")
     def run():
         step.run(d["x_t"], d["v"], d["ref"], dq, dk, dv, t, scale, dt, dt_u)
     step.o_full.fill_(0)
