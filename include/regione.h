@@ -23,6 +23,10 @@
  *    REGIONE_DEV_BOUNDS or REGIONE_DEV_TIMEOUT if a kernel meets an index or
  *    count outside its capacity or a bounded wait runs out.  Kernels never
  *    trap: the offending access is skipped and the kernel ends normally.
+ *  - Kernels are launched with programmatic stream serialization and begin with
+ *    a dependency wait: the order of work on `stream` is exactly that of
+ *    ordinary launches (also under stream capture), only the launch of a kernel
+ *    overlaps the tail of the kernel before it.
  *  - B is the number of independent edit requests in the batch; they share
  *    the sampler schedule (t, dt, scale are scalars).
  *  - There is no CPU fallback: without a CUDA device every compute entry point

@@ -319,3 +319,36 @@ def test_attention_with_scattered_output_rows(counts, D):
     assert int(st[0]) == binding.DEV_BOUNDS
     want[0, rows[0, 0]] = -5.0
     assert torch.equal(got2.view(torch.int16), want.view(torch.int16))
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_shapes_every_row(seed):
+    """Seeded random batches (request count, heads, head size, query / fresh / cached counts, capacities
+    above the counts): every row against the oracle.  Exercises whatever plan the counts produce."""
+    rng = np.random.default_rng(1000 + seed)
+    B = int(rng.integers(1, 5))
+    H = int(rng.integers(1, 7))
+    D = int(rng.choice([64, 128]))
+    counts = []
+    for _ in range(B):
+        nq = int(rng.choice([0, 1, 60, 128, 129, 200, 256, 300, 400, 513]))
+        nf = int(rng.choice([0, 1, 100, 128, 300]))
+        nc = int(rng.choice([0, 5, 128, 500, 1000, 1500]))
+        counts.append((nq, nf, nc))
+    cap_q = max(max(c[0] for c in counts), 1) + int(rng.integers(0, 140))
+    cap_f = max(max(c[1] for c in counts), 1) + int(rng.integers(0, 140))
+    cap_c = max(max(c[2] for c in counts), 1) + int(rng.integers(0, 300))
+    q = _rand_bf16(rng, (B, cap_q, H, D), 0.5)
+    kf, vf = _rand_bf16(rng, (B, cap_f, H, D), 0.5), _rand_bf16(rng, (B, cap_f, H, D))
+    kc, vc = _rand_bf16(rng, (B, cap_c, H, D), 0.5), _rand_bf16(rng, (B, cap_c, H, D))
+    n_q, n_f, n_c = (np.array([c[i] for c in counts], np.int32) for i in range(3))
+    got = run_attention(q, kf, vf, kc, vc, n_q, n_f, n_c, poison=float("nan"))
+    want = orc.region_attention(q, kf, vf, kc, vc, n_q, n_f, n_c, None)
+    for b in range(B):
+        assert np.all(got[b, n_q[b]:] == -3.0), "rows past n_q were written"
+        if n_q[b] == 0:
+            continue
+        if n_f[b] + n_c[b] == 0:
+            assert np.all(got[b, :n_q[b]] == 0.0)          # no key at all: the rows are zero
+        else:
+            assert_close(got[b, :n_q[b]], want[b, :n_q[b]], f"seed {seed} request {b} {counts[b]} H={H} D={D}")
