@@ -63,7 +63,7 @@ constexpr int kAttnThreads = 384;        // 2 softmax warpgroups + 1 of producer
 constexpr int kBM = 128;                 // query rows per tile
 constexpr int kBN = 128;                 // key rows per shared-memory tile
 constexpr int kBH = 64;                  // key rows per P chunk (half a tile)
-constexpr int kPolyEvery = 2;             // every kPolyEvery-th pair computes one of its two exponentials on the FMA pipe
+constexpr int kPolyEvery = 4;             // one pair in kPolyEvery computes one of its two exponentials on the FMA pipe
 constexpr int kHalfBytes = 128 * 64 * 2; // one 128-row x 64-column bf16 box (128-byte rows)
 constexpr long long kTimeoutCycles = 4000000000LL;
 
@@ -344,7 +344,7 @@ __device__ __forceinline__ float chunk_probabilities(uint32_t tP, const uint32_t
 #pragma unroll
     for (int i = 0; i < kBH / 2; ++i) {
         const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, -m));
-        const float p1 = (i % kPolyEvery == 0) ? poly_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m))
+        const float p1 = (i % kPolyEvery == 1) ? poly_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m))
                                                : fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, -m));
         sum[i & 3] += p0 + p1;
         pk[i] = pack_bf16x2(p0, p1);
