@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the attention kernel uses:
-// mbarrier, TMA tiled loads (no multicast anywhere), tcgen05 MMA with tensor
+// mbarrier, TMA tiled loads (every CTA fetches its own tiles), tcgen05 MMA with tensor
 // memory, tensor-memory loads/stores, and the proxy / tcgen05 fences.
 #pragma once
 
