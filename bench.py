@@ -336,7 +336,7 @@ def run_ours(args):
         dist.barrier()
     binding.load()
 
-    steps = 1000 if args.steps is None else args.steps
+    steps = 3000 if args.steps is None else args.steps
     warmup = 10 if args.warmup is None else max(3, args.warmup)
     cfg = args.config
     # weak scaling: every rank owns its own request(s) (a different seed stream), no exchange
