@@ -48,7 +48,7 @@ def measured_peaks():
 
 # DRAM bytes per attention launch on config 2, from the ncu capture summarised in
 # profiles/region_attention_tc_config2.md, valid for the kernel source with this digest only.
-ATTENTION_TRAFFIC = dict(source_sha256_16="31a939943bd5d769", config=2, dram_bytes_per_launch=204.3e6)
+ATTENTION_TRAFFIC = dict(source_sha256_16="c5d947cbeab9fb60", config=2, dram_bytes_per_launch=204.3e6)
 
 
 def recorded_traffic(cfg):

@@ -35,15 +35,17 @@
 //
 // Scheduling: the kernel is persistent, one CTA per SM.  A "step" is one key tile of one
 // (request, head, query pair) item; all steps of the launch form one sequence, item after item,
-// laid out on a cost axis (a step of a pair with one live query tile costs a little less than a
-// step of a full pair, and every item starts with a fixed cost for draining and refilling the
-// pipeline), which is cut into equal contiguous shares, one per CTA (a stream-K decomposition:
+// laid out on a cost axis (a step of a pair with one live query tile costs half a step of a full
+// pair, and every item starts with a fixed cost for draining and refilling the pipeline), which is cut into equal contiguous shares, one per CTA (a stream-K decomposition:
 // the grid is always one balanced wave, whatever the number of items).  A CTA's share is a few
 // segments, each a run of key tiles of one item.  A segment that covers its item completely writes
 // the output rows directly; otherwise it writes its unnormalised output and (max, sum) pair to a
-// slot of the caller's workspace and a small second kernel merges the slots of such items.  The
-// share length is bounded below so that no item is spread over more slots than the workspace
-// holds.  Counts live in device memory, so every CTA derives the same plan from them.
+// slot of the caller's workspace and a small second kernel merges the slots of such items (the
+// attention kernel leaves it a table of the items that its share boundaries cut).  The share
+// length is bounded below so that no item is spread over more slots than the workspace holds.
+// Counts live in device memory, so every CTA derives the same plan from them.  Output rows go to
+// out[b, i] or, with a row list, to out[b, out_rows[b, i]] (the scatter of the attention rows back
+// into the joint sequence, done by whichever kernel writes the row).
 //
 // Every wait is bounded: if a barrier does not complete within ~2 s the CTA
 // records REGIONE_DEV_TIMEOUT, all roles leave their loops, tensor memory is
