@@ -13,7 +13,8 @@ Pins (see tests, marker "not gpu"): straight-line identity, Euler invariance,
 planted-mask recovery, index invariants, scatter(gather) round trip, plain
 copy for the identity keep list, brute-force loops on tiny shapes, agreement
 with a library softmax-attention, split/permutation invariance, uniform-key
-mean, dominant-key selection, the gamma = 1 closed form of the appendix, planted
+mean, dominant-key selection, the row-membership counts and partition-of-the-sequence
+property, the gamma = 1 closed form of the appendix, planted
 decay corrections for the gamma fit, and the zero-edit / full-edit merge cases.
 Every function has such a pin.  Two of them implement a *reading* where the paper
 leaves the operator open, and are pinned as operators only, not against the paper:
@@ -215,6 +216,41 @@ def rikv_store(k_full, v_full, keep_rows, n_keep):
     keep_rows [B, cap]; returns (k_cache, v_cache) [B, cap, H, D], NaN past n_keep[b].
     """
     return gather(k_full, keep_rows, n_keep), gather(v_full, keep_rows, n_keep)
+
+
+# ----------------------------------------------------------------------------
+# Which rows of the joint sequence are recomputed and which come from the cache
+# ----------------------------------------------------------------------------
+
+
+def region_rows(mask, n_text, n_ref, membership="edited_queries"):
+    """Row lists into the joint sequence [text | image | reference] for one request.
+
+    Region-Aware Generation paragraph, the attention equation: the recomputed
+    tokens supply the queries and the fresh keys / values, every other token is
+    served from the Region-Instruction KV cache.
+      ``paper``          : Q = [Q_P, Q_E], fresh = [P, E], cache = [U, I] (the equation as printed:
+                           prompt and edited tokens are recomputed; unedited and instruction-image
+                           tokens are cached).
+      ``edited_queries`` : only the edited image tokens are recomputed; prompt, unedited and
+                           instruction-image tokens all come from the cache.
+    Inside each group rows ascend, and groups are concatenated in joint-sequence order.
+    Returns dict(query, fresh, cache) of int32 arrays.
+    """
+    m = np.asarray(mask).astype(bool).reshape(-1)
+    n_img = m.shape[0]
+    query, cache = [], []
+    recompute_text = {"paper": True, "edited_queries": False}[membership]
+    for row in range(n_text + n_img + n_ref):
+        if row < n_text:
+            recomputed = recompute_text
+        elif row < n_text + n_img:
+            recomputed = bool(m[row - n_text])
+        else:
+            recomputed = False
+        (query if recomputed else cache).append(row)
+    q = np.asarray(query, np.int32)
+    return dict(query=q, fresh=q.copy(), cache=np.asarray(cache, np.int32))
 
 
 # ----------------------------------------------------------------------------

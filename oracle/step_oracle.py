@@ -2,13 +2,20 @@
 
 TEST INFRASTRUCTURE ONLY (same rules as regione_oracle).  Mirrors Algorithm 1 for one layer:
 partition, gather, cache store, region attention, scatter, velocity decay + Euler, merge.
+``wl`` is only read for its shape fields (batch, n_text, n_ref, metric, threshold); nothing of the
+product package is imported.
+
+Pins (marker "not gpu", tests/test_oracle_step.py): a zero-edit mask gives x - dt_U * v on every token
+and an all-zero attention output; a full mask under the paper's membership with no reference tokens
+reduces the attention rows to a library softmax attention; the counts of the tiny configuration;
+edited tokens of the merged latent equal X^E after the Euler step and unedited ones lie on the
+straight line; the cache holds exactly the rows the membership rule names.
 """
 from __future__ import annotations
 
 import numpy as np
 
 from oracle import regione_oracle as orc
-from paper_2510_25590_b200 import synth
 
 
 def region_step(wl, lat, qkv, t, scale, dt, dt_unedited, membership="edited_queries", heads=None):
@@ -20,7 +27,7 @@ def region_step(wl, lat, qkv, t, scale, dt, dt_unedited, membership="edited_quer
     metric = orc.COSINE if wl.metric == "cosine" else orc.L2
     B = wl.batch
     p = orc.partition(lat["x_t"], lat["v"], lat["ref"], t, metric, wl.threshold)
-    rows = [synth.region_rows(wl, p["mask"][b], membership) for b in range(B)]
+    rows = [orc.region_rows(p["mask"][b], wl.n_text, wl.n_ref, membership) for b in range(B)]
     nq = np.array([len(r["query"]) for r in rows], np.int32)
     nc = np.array([len(r["cache"]) for r in rows], np.int32)
     q_cap, c_cap = max(1, int(nq.max())), max(1, int(nc.max()))

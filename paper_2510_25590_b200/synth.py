@@ -291,29 +291,6 @@ def make_qkv_full(wl: Workload, *, stream: int = 0, std: float | None = None):
     return out
 
 
-def region_rows(wl: Workload, mask: np.ndarray, membership: str = "edited_queries"):
-    """Row lists (into the joint sequence) for one batch entry's region-attention call.
-
-    ``edited_queries``: queries and fresh K/V are the edited image tokens; the
-    cache holds text, unedited image and reference tokens.
-    ``paper``: queries and fresh K/V are [text, edited] (the attention equation
-    of the Region-Aware Generation paragraph); the cache holds [unedited, reference].
-    Rows are ascending inside each group.
-    """
-    Tt, N, Nr = wl.n_text, wl.n_img, wl.n_ref
-    m = np.asarray(mask).astype(bool)
-    img = np.arange(N, dtype=np.int32) + Tt
-    text = np.arange(Tt, dtype=np.int32)
-    refr = np.arange(Nr, dtype=np.int32) + Tt + N
-    edited, unedited = img[m], img[~m]
-    if membership == "edited_queries":
-        return dict(query=edited, fresh=edited, cache=np.concatenate([text, unedited, refr]))
-    if membership == "paper":
-        pe = np.concatenate([text, edited])
-        return dict(query=pe, fresh=pe, cache=np.concatenate([unedited, refr]))
-    raise ValueError(membership)
-
-
 # ----------------------------------------------------------------------------
 # sampler schedule inputs
 # ----------------------------------------------------------------------------

@@ -58,7 +58,7 @@ def region_case(wl, ratio=None, membership="edited_queries", std=None, stream=0)
     lat_mask = synth.make_latents(wl, ratio)["mask"]
     qkv = synth.make_qkv_full(wl, stream=stream, std=std)
     B = wl.batch
-    rows = [synth.region_rows(wl, lat_mask[b], membership) for b in range(B)]
+    rows = [orc.region_rows(lat_mask[b], wl.n_text, wl.n_ref, membership) for b in range(B)]
     nq = np.array([len(r["query"]) for r in rows], np.int32)
     nf = np.array([len(r["fresh"]) for r in rows], np.int32)
     nc = np.array([len(r["cache"]) for r in rows], np.int32)

@@ -146,7 +146,7 @@ def test_morphological_open_close_matches_oracle():
 
 
 @pytest.mark.parametrize("membership", ["edited_queries", "paper"])
-def test_region_rows_match_generator_layout(membership):
+def test_region_rows_match_the_oracle_membership_rule(membership):
     import torch
     wl = synth.scaled_workload(synth.WORKLOADS[5], grid=(48, 48), n_text=77, batch=3)
     lat = synth.make_latents(wl)
@@ -163,7 +163,7 @@ def test_region_rows_match_generator_layout(membership):
     torch.cuda.synchronize()
     assert int(st[0]) == 0
     for b in range(B):
-        want = synth.region_rows(wl, p["mask"][b], membership)
+        want = orc.region_rows(p["mask"][b], wl.n_text, wl.n_ref, membership)
         assert int(nq[b]) == len(want["query"]) and int(nc[b]) == len(want["cache"])
         assert np.array_equal(qr[b, :int(nq[b])].cpu().numpy(), want["query"])
         assert np.array_equal(cr[b, :int(nc[b])].cpu().numpy(), want["cache"])
@@ -174,7 +174,7 @@ def test_region_rows_match_generator_layout(membership):
 @pytest.mark.parametrize("grid,n_text,batch", [((48, 48), 77, 3), ((64, 64), 512, 1), ((9, 7), 0, 2), ((96, 96), 33, 2)])
 def test_partition_with_row_lists_in_one_launch(membership, grid, n_text, batch):
     """regione_partition_rows = regione_partition + regione_region_rows: every output bit-exact
-    against the oracle partition and the generator's row layout, tails untouched."""
+    against the oracle partition and the oracle row lists, tails untouched."""
     import torch
     wl = synth.scaled_workload(synth.WORKLOADS[5], grid=grid, n_text=n_text, batch=batch)
     lat = synth.make_latents(wl)
@@ -200,7 +200,7 @@ def test_partition_with_row_lists_in_one_launch(membership, grid, n_text, batch)
                slot=s.cpu().numpy(), n_edit=ne.cpu().numpy(), score=score.cpu().numpy())
     check_against_oracle(got, p, N)
     for b in range(B):
-        want = synth.region_rows(wl, p["mask"][b], membership)
+        want = orc.region_rows(p["mask"][b], wl.n_text, wl.n_ref, membership)
         assert int(nq[b]) == len(want["query"]) and int(nc[b]) == len(want["cache"])
         assert np.array_equal(qr[b, :int(nq[b])].cpu().numpy(), want["query"])
         assert np.array_equal(cr[b, :int(nc[b])].cpu().numpy(), want["cache"])
