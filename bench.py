@@ -46,8 +46,8 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-# DRAM bytes per attention launch on config 2, from the ncu capture summarised in
-# profiles/region_attention_tc_config2.md, valid for the kernel source with this digest only.
+# DRAM bytes per attention launch on config 2 (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture of this workload), valid for the kernel source with this digest only.
 ATTENTION_TRAFFIC = dict(source_sha256_16="c5d947cbeab9fb60", config=2, dram_bytes_per_launch=204.3e6)
 
 
@@ -282,7 +282,8 @@ def hbm_sweep(torch, binding, step, d, flush_l2, peak_gbs, iters=10):
 
 def ratio_sweep(torch, binding, synth, flush_l2, to_dev, steps=20):
     """Denoise-step time against the edit-mask ratio on the Qwen-Image-Edit-shaped workload (config 3):
-    one region step (all 12 calls) and its attention call per ratio, CUDA events, L2 flushed per step."""
+    one region step (7 library calls, 8 launches) and its attention call per ratio, CUDA events, L2
+    flushed per step."""
     from paper_2510_25590_b200.step import RegionStep, StepShapes, plan_capacity
     wl = synth.WORKLOADS[3]
     qkv = synth.make_qkv_full(wl)
@@ -314,6 +315,141 @@ def ratio_sweep(torch, binding, synth, flush_l2, to_dev, steps=20):
                         attention_tflops=round(fl / at_us / 1e6, 1)))
         del step
     return out
+
+
+def per_config_rows(torch, binding, synth, flush_l2, to_dev, peaks, steps=12):
+    """The other configurations beside the headline one, each timed like it (CUDA events, L2 flushed
+    before every step): the tiny layer (config 1), the Step1X-Edit-shaped attention layer with the
+    paper's membership and the L2 partition (config 4's shape) and the batch of four large requests
+    (config 5); then config 4's 28-step loop, library calls only."""
+    from paper_2510_25590_b200.step import RegionStep, StepShapes, plan_capacity
+    rows = []
+    for cfg, membership in ((1, "edited_queries"), (4, "paper"), (5, "edited_queries")):
+        wl = synth.WORKLOADS[cfg]
+        lat = synth.make_latents(wl)
+        qkv = synth.make_qkv_full(wl)
+        x_t, v, ref = (to_dev(lat[k]) for k in ("x_t", "v", "ref"))
+        dq, dk, dv = (to_dev(qkv[k]) for k in ("q", "k", "v"))
+        del qkv
+        metric = binding.METRIC_COSINE if wl.metric == "cosine" else binding.METRIC_L2
+        cap = plan_capacity(x_t, v, ref, lat["t"], metric, wl.threshold)
+        step = RegionStep(StepShapes(wl.batch, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads,
+                                     wl.head_dim, cap, metric, wl.threshold,
+                                     binding.ROWS_PAPER if membership == "paper" else binding.ROWS_EDITED_QUERIES))
+        run = lambda: step.run(x_t, v, ref, dq, dk, dv, lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0)
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+        for i in range(steps):
+            flush_l2()
+            step.attention_events = (ev[i][1], ev[i][2])
+            ev[i][0].record(); run(); ev[i][3].record()
+        torch.cuda.synchronize()
+        step.attention_events = None
+        assert int(step.dev_status[0]) == 0
+        n_q = step.n_q.cpu().numpy(); n_kv = n_q + step.n_cache.cpu().numpy()
+        fl = attention_flops(n_q, n_kv, wl.heads, wl.head_dim)
+        st_us = float(np.mean([e[0].elapsed_time(e[3]) for e in ev]) * 1e3)
+        at_us = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]) * 1e3)
+        tf = fl / at_us / 1e6
+        rows.append(dict(config=cfg, workload=wl.name, membership=membership, batch=wl.batch,
+                         n_q=int(n_q[0]), n_kv=int(n_kv[0]), heads=wl.heads, head_dim=wl.head_dim,
+                         step_us=round(st_us, 1), attention_us=round(at_us, 1), attention_tflops=round(tf, 1),
+                         attention_frac_of_measured_burst=round(tf / peaks["bf16_tflops"], 3),
+                         attention_frac_of_nominal_2250=round(tf / NOMINAL_BF16_TFLOPS, 3),
+                         step_tflops_equivalent=round(fl / st_us / 1e6, 1)))
+        del step, dq, dk, dv
+        torch.cuda.empty_cache()
+    rows.append(loop_row(torch, binding, synth, to_dev))
+    return rows
+
+
+def loop_row(torch, binding, synth, to_dev):
+    """Config 4's sampler loop (4096 tokens x 16 channels, L2 partition after step 6, cache refresh every
+    5 steps, alternate region steps reused: 28 steps): device time of the library calls alone.  The
+    velocity model is scaffold around the path, so its outputs are recorded in a first pass and replayed
+    from memory in the timed passes (no model kernel runs inside them); the host decisions depend on the
+    schedule only, so the whole loop is also captured once into a CUDA graph and replayed."""
+    from paper_2510_25590_b200 import loop as gloop
+    wl = synth.WORKLOADS[4]
+    lat = synth.make_latents(wl, stream=4)
+    rng = np.random.default_rng(4)
+    m = lat["mask"].astype(bool)
+    ref_h = lat["ref"]
+    target = to_dev(synth.bf16_round(np.where(m[..., None], rng.standard_normal(ref_h.shape), ref_h).astype(np.float32))).float()
+    noise = to_dev(synth.bf16_round(rng.standard_normal(ref_h.shape).astype(np.float32)))
+    ref = to_dev(ref_h)
+    kinds, after = gloop.alternating_schedule()
+    T = len(kinds)
+    ts = [1.0 - k / T for k in range(T + 1)]
+    cfg = gloop.LoopConfig(kinds, after, ts, [1.0] * (T + 1), 0.05, binding.METRIC_L2, wl.threshold)
+    B, N, C = noise.shape
+    lp = gloop.RegionELoop(B, N, C, cfg)
+
+    class Recording:
+        def __init__(self):
+            self.full_out, self.region_out = [], []
+
+        def full(self, x, t, store):
+            self.full_out.append(((x.float() - target) / t).to(x.dtype))
+            return self.full_out[-1]
+
+        def region(self, x_e, t, edit_idx, n_edit):
+            idx = edit_idx.long().clamp(0, N - 1)
+            tgt = torch.gather(target, 1, idx.unsqueeze(-1).expand(B, x_e.shape[1], C))
+            self.region_out.append(((x_e.float() - tgt) / t).to(x_e.dtype))
+            return self.region_out[-1]
+
+    class Replay:
+        def __init__(self, rec):
+            self.rec, self.i, self.j = rec, 0, 0
+
+        def full(self, x, t, store):
+            self.i += 1
+            return self.rec.full_out[self.i - 1]
+
+        def region(self, x_e, t, edit_idx, n_edit):
+            self.j += 1
+            return self.rec.region_out[self.j - 1]
+
+    rec = Recording()
+    x = noise.clone()
+    _, trace = lp.run(x, ref, rec)
+    torch.cuda.synchronize()
+    assert int(lp.dev_status[0]) == 0
+
+    def replay_once():
+        x.copy_(noise)
+        return lp.run(x, ref, Replay(rec))
+
+    eager = []
+    for i in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        x.copy_(noise)
+        a.record(); lp.run(x, ref, Replay(rec)); b.record()
+        torch.cuda.synchronize()
+        eager.append(a.elapsed_time(b) * 1e3)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            lp.run(x, ref, Replay(rec), stream=side)
+    torch.cuda.synchronize()
+    graphed = []
+    for i in range(10):
+        x.copy_(noise)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); graph.replay(); b.record()
+        torch.cuda.synchronize()
+        graphed.append(a.elapsed_time(b) * 1e3)
+    n_reuse = sum(1 for s_ in trace.steps if s_[2] == "reuse")
+    return dict(config=4, workload=wl.name + ": 28-step loop, library calls only", schedule=kinds,
+                image_tokens=N, channels=C, full_steps=kinds.count("F"), region_steps=kinds.count("R"),
+                reused_region_steps=n_reuse, library_launches=trace.launches,
+                loop_us_eager_python=round(float(np.median(eager)), 1),
+                loop_us_cuda_graph=round(float(np.median(graphed)), 1),
+                us_per_launch_cuda_graph=round(float(np.median(graphed)) / max(trace.launches, 1), 2))
 
 
 def run_ours(args):
@@ -459,11 +595,15 @@ def run_ours(args):
     step_vs_ratio = None
     if world == 1 and not args.no_ratio_sweep:
         step_vs_ratio = ratio_sweep(torch, binding, synth, flush_l2, dev)
+    per_config = None
+    if world == 1 and not args.no_per_config:
+        per_config = per_config_rows(torch, binding, synth, flush_l2, dev, peaks)
     attn_us = float(np.mean(attn_ms) * 1e3)
     achieved = flops / (attn_us * 1e-6) / 1e12
     roofline = dict(bound="tensor", achieved=achieved, peak=peaks["bf16_tflops"], unit="TFLOP/s",
                     frac=achieved / peaks["bf16_tflops"], traffic=recorded_traffic(cfg),
-                    kernel="region_attention_tc_kernel<128>", us_per_launch=attn_us,
+                    kernel=f"region_attention_tc_kernel<{wl.head_dim}> (+ merge of shared items)",
+                    us_per_launch=attn_us,
                     peak_source=f"bf16_tflops (burst) of {peaks['source']}",
                     frac_of_nominal_2250=achieved / NOMINAL_BF16_TFLOPS)
 
@@ -487,7 +627,7 @@ def run_ours(args):
                 e2e=dict(value=e2e_val, unit=UNIT, h2d_bytes_per_step=int(h2d), d2h_bytes_per_step=int(d2h),
                          steps=e2e_steps, ms_per_step=e2e_ms / e2e_steps),
                 gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu_baseline,
-                hbm_kernels=hbm_kernels, denoise_step_us_vs_mask_ratio=step_vs_ratio,
+                hbm_kernels=hbm_kernels, denoise_step_us_vs_mask_ratio=step_vs_ratio, per_config=per_config,
                 step_us=dict(mean=float(step_ms.mean() * 1e3), min=float(step_ms.min() * 1e3),
                              median=float(np.median(step_ms) * 1e3)),
                 attention_us=dict(mean=attn_us, min=float(attn_ms.min() * 1e3)),
@@ -507,6 +647,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-hbm-sweep", action="store_true")
     ap.add_argument("--no-ratio-sweep", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

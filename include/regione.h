@@ -23,12 +23,17 @@
  *    REGIONE_DEV_BOUNDS or REGIONE_DEV_TIMEOUT if a kernel meets an index or
  *    count outside its capacity or a bounded wait runs out.  Kernels never
  *    trap: the offending access is skipped and the kernel ends normally.
- *  - Kernels are launched with programmatic stream serialization and begin with
- *    a dependency wait: the order of work on `stream` is exactly that of
- *    ordinary launches (also under stream capture), only the launch of a kernel
- *    overlaps the tail of the kernel before it.
- *  - B is the number of independent edit requests in the batch; they share
- *    the sampler schedule (t, dt, scale are scalars).
+ *  - Every kernel of the product entry points is launched with programmatic
+ *    stream serialization and begins with a dependency wait: the order of work
+ *    on `stream` is exactly that of ordinary launches (also under stream
+ *    capture), only the launch of a kernel overlaps the tail of the kernel
+ *    before it.  The two entry points of the "cross-check and self-test"
+ *    section at the end are ordinary launches.
+ *  - B is the number of independent edit requests in the batch.  Each request
+ *    may sit at its own sampler step: the sampler scalars (t, dt, scale,
+ *    dt_unedited) are host arrays of B floats, read during the call (the
+ *    values travel to the kernels as launch parameters, 128 requests per
+ *    launch; the arrays may be reused as soon as the call returns).
  *  - There is no CPU fallback: without a CUDA device every compute entry point
  *    returns REGIONE_CUDA_ERROR.
  */
@@ -79,15 +84,16 @@ const char* regione_status_string(int status);
  * A zero cosine denominator is clamped at 1e-12.
  *
  * x_t, v, ref : dev bf16 [B, N, C], C a multiple of 8 and <= 4096
+ * t           : host f32 [B], the sampler time of each request
  * mask        : dev u8    [B, N]   (1 = edited)
  * edit_idx, keep_idx, slot : dev int32 [B, N]; entries of edit_idx / keep_idx past
  *               the live prefix are left untouched
  * n_edit      : dev int32 [B]
  * score       : dev f32   [B, N], nullable; receives s
- * Limits: 1 <= N <= 2^21 per request, B <= 65535.
+ * Limits: 1 <= N <= 2^20 per request (REGIONE_UNSUPPORTED above), B <= 65535.
  */
 int regione_partition(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
-                      int B, int N, int C, float t, int metric, float threshold,
+                      int B, int N, int C, const float* t, int metric, float threshold,
                       uint8_t* mask, int32_t* edit_idx, int32_t* keep_idx, int32_t* slot,
                       int32_t* n_edit, float* score, int32_t* dev_status, void* stream);
 
@@ -100,7 +106,7 @@ int regione_partition(const regione_bf16* x_t, const regione_bf16* v, const regi
  * second launch and its pass over the lists are saved.
  */
 int regione_partition_rows(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
-                           int B, int N, int C, float t, int metric, float threshold,
+                           int B, int N, int C, const float* t, int metric, float threshold,
                            uint8_t* mask, int32_t* edit_idx, int32_t* keep_idx, int32_t* slot,
                            int32_t* n_edit, float* score,
                            int n_text, int n_ref, int membership,
@@ -110,11 +116,13 @@ int regione_partition_rows(const regione_bf16* x_t, const regione_bf16* v, const
 
 /*
  * Morphological opening then closing of the edited mask on the rows x cols token
- * grid (Sec. 4, "Adaptive Region Partition": "morphological opening and closing
- * operations"; Algorithm 1 calls it Erosion_&_Dilate), followed by the same
- * compaction as regione_partition.  Structuring element 3x3; neighbours outside
- * the grid are ignored.  mask_in [B, rows*cols] -> mask_out and the index lists.
+ * grid (Sec. 4, "Adaptive Region Partition", the clean-up that makes the two
+ * regions more contiguous; Algorithm 1 names an erosion and a dilation), followed
+ * by the same compaction as regione_partition.  Structuring element 3x3; neighbours
+ * outside the grid are ignored.  mask_in [B, rows*cols] -> mask_out and the index lists.
  * mask_in and mask_out may not alias.  rows*cols <= 16384.
+ * dev_status is accepted for uniformity and never written: the kernel has no count
+ * or index input that could be out of range on the device.
  */
 int regione_mask_open_close(const uint8_t* mask_in, int B, int rows, int cols,
                             uint8_t* mask_out, int32_t* edit_idx, int32_t* keep_idx,
@@ -163,8 +171,9 @@ int regione_gather_multi(const void* const* srcs, void* const* dsts, int n_tenso
                          int32_t* dev_status, void* stream);
 
 /*
- * Token scatter, the inverse placement (Sec. 4: results are "re-gathered according
- * to their spatial positions"; Algorithm 1, the gather(...) line):
+ * Token scatter, the inverse placement (Sec. 4, end of the AVDCache paragraph: the
+ * region results are put back at their spatial positions; Algorithm 1, the
+ * gather(...) line):
  *     dst[b, idx[b, j], :] = src[b, j, :]     for j < min(n[b], src_rows_cap)
  * Other rows of dst are left untouched.  idx must not repeat a row.
  */
@@ -255,15 +264,18 @@ int regione_region_attention_scatter(const regione_bf16* q,
  * start-up so a later cudaMalloc fails, or a denoising loop that must not stall,
  * since cudaMalloc / cudaFree synchronise the whole device.  The split-KV partials
  * go to a 64 MiB array compiled into the library (device memory that every GPU
- * loading the library holds until the process ends); the call performs no
- * allocation of any kind.
+ * loading the library holds until the process ends); the call itself requests no
+ * memory from the CUDA runtime or any other allocator.
  *
  *  - A shape whose partials would not fit, i.e.
  *    regione_region_attention_workspace(...) > 64 MiB, is refused with
  *    REGIONE_WORKSPACE_TOO_SMALL; nothing is launched.
  *  - The first call on each device looks the array's device address up (with that
  *    device current) and remembers it.  Make that first call outside any stream
- *    capture.
+ *    capture.  Under the CUDA runtime's lazy module loading that first use is also
+ *    the moment the driver places the library's device image, array included, in
+ *    device memory: make one warm-up call per device at start-up, BEFORE an arena
+ *    takes the rest of HBM, or the warm-up itself fails with REGIONE_CUDA_ERROR.
  *  - All calls on a device share the one array and it keeps whatever the last call
  *    left in it.  Nothing in it needs clearing between calls, but two calls whose
  *    kernels overlap on the GPU (different streams) race on it: serialise them.
@@ -287,8 +299,8 @@ int regione_avd_step(double* running_product, double dt, double gamma, double de
 
 /*
  * Fit of the timestep-aware decay correction gamma (Sec. 4, "Adaptive Velocity Decay
- * Cache", decay-factor equation: ||v_{t_i}|| / ||v_{t_{i+1}}|| = (1 - dt_i) * gamma_{t_i},
- * gamma "obtained by fitting on a randomly sampled dataset").  From the velocities of S
+ * Cache", decay-factor equation: ||v_{t_i}|| / ||v_{t_{i+1}}|| = (1 - dt_i) * gamma_{t_i};
+ * the paper fits gamma on sampled data).  From the velocities of S
  * sampled trajectories at T1 consecutive steps:
  *     norms[s, i] = || v[s, i, :] ||_2
  *     gamma[i]    = mean_s( norms[s, i] / norms[s, i+1] ) / (1 - dt[i]),     i < T1 - 1
@@ -303,14 +315,15 @@ int regione_gamma_fit(const regione_bf16* v, int S, int T1, int64_t n, const flo
 /*
  * Decayed cached velocity and Euler update of the edited tokens (Sec. 4, the
  * case equation of the AVDCache; Sec. 3, the Euler sampler equation):
- *     v_use = scale * v_in[b,j,:]
- *     x_e[b,j,:] <- x_e[b,j,:] - dt * v_use                for j < n_edit[b]
+ *     v_use = scale[b] * v_in[b,j,:]
+ *     x_e[b,j,:] <- x_e[b,j,:] - dt[b] * v_use             for j < n_edit[b]
  *     v_cache_out[b,j,:] <- v_in[b,j,:]   (if v_cache_out != NULL: a recomputed step
  *                                          refreshes the velocity cache)
- * scale is the accumulated decay product on a reused step and 1 on a recomputed one.
+ * scale[b] is the accumulated decay product on a reused step and 1 on a recomputed one.
  * v_in, x_e, v_cache_out : dev bf16 [B, Ne_cap, C], C a multiple of 8.
+ * scale, dt : host f32 [B] (requests of one batch may sit at different sampler steps).
  */
-int regione_velocity_decay(const regione_bf16* v_in, float scale, float dt, regione_bf16* x_e,
+int regione_velocity_decay(const regione_bf16* v_in, const float* scale, const float* dt, regione_bf16* x_e,
                            regione_bf16* v_cache_out, const int32_t* n_edit,
                            int B, int Ne_cap, int C, int32_t* dev_status, void* stream);
 
@@ -319,14 +332,48 @@ int regione_velocity_decay(const regione_bf16* v_in, float scale, float dt, regi
  * estimation equation applied to the unedited tokens; Algorithm 1, the one-step
  * line before the inner loop and the gather line after it):
  *     x_out[b,n,:] = slot[b,n] >= 0 ? x_e[b, slot[b,n], :]
- *                                   : x_full[b,n,:] - dt_unedited * v_last_full[b,n,:]
- * x_full, v_last_full, x_out : dev bf16 [B, N, C]; x_e [B, Ne_cap, C]; slot dev int32 [B, N].
- * x_out may alias x_full.  A slot >= Ne_cap is skipped and REGIONE_DEV_BOUNDS recorded.
+ *                                   : x_full[b,n,:] - dt_unedited[b] * v_last_full[b,n,:]
+ * x_full, v_last_full, x_out : dev bf16 [B, N, C]; x_e [B, Ne_cap, C]; slot dev int32 [B, N];
+ * dt_unedited host f32 [B].  x_out may alias x_full.  A slot >= Ne_cap is skipped and REGIONE_DEV_BOUNDS recorded.
  */
 int regione_merge(const regione_bf16* x_full, const regione_bf16* v_last_full,
-                  const regione_bf16* x_e, const int32_t* slot, float dt_unedited,
+                  const regione_bf16* x_e, const int32_t* slot, const float* dt_unedited,
                   int B, int N, int Ne_cap, int C, regione_bf16* x_out,
                   int32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Cross-check and self-test entry points.  Test infrastructure that has to live inside the
+ * library because it runs on the device; no product entry point above calls either of them,
+ * and both are ordinary (not dependency-wait) launches.
+ * ------------------------------------------------------------------------------------------ */
+
+/*
+ * The attention equation of Sec. 4 "Region-Aware Generation" once more, on the CUDA cores: one
+ * warp per (request, head, query row), fp32 online softmax, no tensor cores, no shared plan.
+ * Same arguments, layouts and results as regione_region_attention minus the workspace.  It is
+ * orders of magnitude slower and exists so that tests can compare the tensor-core kernel with
+ * an independent arithmetic path on the same device at sizes where the CPU oracle is slow.
+ */
+int regione_crosscheck_region_attention(const regione_bf16* q,
+                                        const regione_bf16* k_fresh, const regione_bf16* v_fresh,
+                                        const regione_bf16* k_cache, const regione_bf16* v_cache,
+                                        const int32_t* n_q, const int32_t* n_fresh, const int32_t* n_cache,
+                                        int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D,
+                                        float softmax_scale, regione_bf16* out,
+                                        int32_t* dev_status, void* stream);
+
+/*
+ * Lets a bounded wait run out, in the harmless form (the paper has no counterpart; this covers
+ * the convention above that a wait that expires ends in REGIONE_DEV_TIMEOUT).  One thread of one
+ * thread block waits, through the very routine the attention kernel's roles wait with, on a
+ * barrier that nothing ever arrives on, with no copy and no tensor-core operation in flight.
+ * After limit_cycles SM clock cycles (1 .. 10^8) the wait gives up, REGIONE_DEV_TIMEOUT is
+ * recorded in dev_status and the kernel ends normally; the context stays usable.
+ * out : dev int64 [3], nullable: {1 if the wait claimed completion (must be 0), cycles spent
+ *       waiting, the abort flag the other roles would have seen (must be 1)}.
+ */
+int regione_selftest_bounded_wait(long long limit_cycles, int32_t* dev_status, long long* out,
+                                  void* stream);
 
 #ifdef __cplusplus
 }

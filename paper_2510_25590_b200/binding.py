@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, c_char_p, c_double, c_float, c_int, c_int64, c_size_t, c_void_p
+from ctypes import POINTER, c_char_p, c_double, c_float, c_int, c_int64, c_longlong, c_size_t, c_void_p
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libregione.so")
@@ -24,9 +24,9 @@ _P = c_void_p
 SIGNATURES = {
     "regione_version": (c_int, []),
     "regione_status_string": (c_char_p, [c_int]),
-    "regione_partition": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_float, c_int, c_float,
+    "regione_partition": (c_int, [_P, _P, _P, c_int, c_int, c_int, _P, c_int, c_float,
                                   _P, _P, _P, _P, _P, _P, _P, _P]),
-    "regione_partition_rows": (c_int, [_P, _P, _P, c_int, c_int, c_int, c_float, c_int, c_float,
+    "regione_partition_rows": (c_int, [_P, _P, _P, c_int, c_int, c_int, _P, c_int, c_float,
                                        _P, _P, _P, _P, _P, _P, c_int, c_int, c_int,
                                        _P, _P, c_int, _P, _P, c_int, _P, _P]),
     "regione_mask_open_close": (c_int, [_P, c_int, c_int, c_int, _P, _P, _P, _P, _P, _P, _P]),
@@ -42,8 +42,10 @@ SIGNATURES = {
     "regione_region_attention_static": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, _P]),
     "regione_avd_step": (c_int, [POINTER(c_double), c_double, c_double, c_double, POINTER(c_int)]),
     "regione_gamma_fit": (c_int, [_P, c_int, c_int, c_int64, _P, _P, _P, _P]),
-    "regione_velocity_decay": (c_int, [_P, c_float, c_float, _P, _P, _P, c_int, c_int, c_int, _P, _P]),
-    "regione_merge": (c_int, [_P, _P, _P, _P, c_float, c_int, c_int, c_int, c_int, _P, _P, _P]),
+    "regione_velocity_decay": (c_int, [_P, _P, _P, _P, _P, _P, c_int, c_int, c_int, _P, _P]),
+    "regione_merge": (c_int, [_P, _P, _P, _P, _P, c_int, c_int, c_int, c_int, _P, _P, _P]),
+    "regione_crosscheck_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, _P]),
+    "regione_selftest_bounded_wait": (c_int, [c_longlong, _P, _P, _P]),
 }
 
 
@@ -107,6 +109,18 @@ def _stream(stream=None):
     return c_void_p(s.cuda_stream)
 
 
+def _per_request(value, B, name):
+    """A sampler scalar for the batch: one number (shared by every request) or B numbers (each
+    request at its own sampler step) -> a host float array of length B."""
+    try:
+        vals = [float(value)] * B
+    except (TypeError, ValueError):
+        vals = [float(x) for x in value]
+        if len(vals) != B:
+            raise RegionEError(f"{name} must be one number or {B} numbers, got {len(vals)}")
+    return (c_float * max(B, 1))(*vals)
+
+
 def version() -> int:
     return load().regione_version()
 
@@ -117,7 +131,8 @@ def partition(x_t, v, ref, t, metric, threshold, mask, edit_idx, keep_idx, slot,
     B, N, C = x_t.shape
     bf = torch.bfloat16
     _check(load().regione_partition(
-        _ptr(x_t, bf, "x_t"), _ptr(v, bf, "v"), _ptr(ref, bf, "ref"), B, N, C, float(t), int(metric),
+        _ptr(x_t, bf, "x_t"), _ptr(v, bf, "v"), _ptr(ref, bf, "ref"), B, N, C, _per_request(t, B, "t"),
+        int(metric),
         float(threshold), _ptr(mask, torch.uint8, "mask"), _ptr(edit_idx, torch.int32, "edit_idx"),
         _ptr(keep_idx, torch.int32, "keep_idx"), _ptr(slot, torch.int32, "slot"),
         _ptr(n_edit, torch.int32, "n_edit"), _ptr(score, torch.float32, "score"),
@@ -132,7 +147,8 @@ def partition_rows(x_t, v, ref, t, metric, threshold, mask, edit_idx, keep_idx, 
     B, N, C = x_t.shape
     bf, i32 = torch.bfloat16, torch.int32
     _check(load().regione_partition_rows(
-        _ptr(x_t, bf, "x_t"), _ptr(v, bf, "v"), _ptr(ref, bf, "ref"), B, N, C, float(t), int(metric),
+        _ptr(x_t, bf, "x_t"), _ptr(v, bf, "v"), _ptr(ref, bf, "ref"), B, N, C, _per_request(t, B, "t"),
+        int(metric),
         float(threshold), _ptr(mask, torch.uint8, "mask"), _ptr(edit_idx, i32, "edit_idx"),
         _ptr(keep_idx, i32, "keep_idx"), _ptr(slot, i32, "slot"), _ptr(n_edit, i32, "n_edit"),
         _ptr(score, torch.float32, "score"), int(n_text), int(n_ref), int(membership),
@@ -282,6 +298,30 @@ def region_attention_static(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh,
         _ptr(dev_status, i32), _stream(stream)), "regione_region_attention_static")
 
 
+def crosscheck_region_attention(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, out,
+                                softmax_scale=0.0, dev_status=None, stream=None):
+    """The CUDA-core statement of the attention equation (test infrastructure, not a product path)."""
+    torch = _torch()
+    bf = torch.bfloat16
+    B, Nq_cap, H, D = q.shape
+    Nf_cap = 0 if k_fresh is None else k_fresh.shape[1]
+    Nc_cap = 0 if k_cache is None else k_cache.shape[1]
+    i32 = torch.int32
+    _check(load().regione_crosscheck_region_attention(
+        _ptr(q, bf, "q"), _ptr(k_fresh, bf, "k_fresh"), _ptr(v_fresh, bf, "v_fresh"),
+        _ptr(k_cache, bf, "k_cache"), _ptr(v_cache, bf, "v_cache"), _ptr(n_q, i32), _ptr(n_fresh, i32),
+        _ptr(n_cache, i32), B, Nq_cap, Nf_cap, Nc_cap, H, D, float(softmax_scale), _ptr(out, bf, "out"),
+        _ptr(dev_status, i32), _stream(stream)), "regione_crosscheck_region_attention")
+
+
+def selftest_bounded_wait(limit_cycles, dev_status, out=None, stream=None):
+    """Lets one bounded wait expire on the device (see the header); ``out`` int64 [3], optional."""
+    torch = _torch()
+    _check(load().regione_selftest_bounded_wait(
+        int(limit_cycles), _ptr(dev_status, torch.int32, "dev_status"), _ptr(out, torch.int64, "out"),
+        _stream(stream)), "regione_selftest_bounded_wait")
+
+
 def avd_step(running_product: float, dt: float, gamma: float, delta: float):
     """Returns (new_running_product, reuse)."""
     p = c_double(running_product)
@@ -306,7 +346,8 @@ def velocity_decay(v_in, scale, dt, x_e, n_edit, v_cache_out=None, dev_status=No
     bf = torch.bfloat16
     B, Ne_cap, C = x_e.shape
     _check(load().regione_velocity_decay(
-        _ptr(v_in, bf, "v_in"), float(scale), float(dt), _ptr(x_e, bf, "x_e"),
+        _ptr(v_in, bf, "v_in"), _per_request(scale, B, "scale"), _per_request(dt, B, "dt"),
+        _ptr(x_e, bf, "x_e"),
         _ptr(v_cache_out, bf, "v_cache_out"), _ptr(n_edit, torch.int32), B, Ne_cap, C,
         _ptr(dev_status, torch.int32), _stream(stream)), "regione_velocity_decay")
 
@@ -317,5 +358,6 @@ def merge(x_full, v_last_full, x_e, slot, dt_unedited, x_out, dev_status=None, s
     B, N, C = x_full.shape
     _check(load().regione_merge(
         _ptr(x_full, bf, "x_full"), _ptr(v_last_full, bf, "v_last_full"), _ptr(x_e, bf, "x_e"),
-        _ptr(slot, torch.int32), float(dt_unedited), B, N, 0 if x_e is None else x_e.shape[1], C,
+        _ptr(slot, torch.int32), _per_request(dt_unedited, B, "dt_unedited"), B, N,
+        0 if x_e is None else x_e.shape[1], C,
         _ptr(x_out, bf, "x_out"), _ptr(dev_status, torch.int32), _stream(stream)), "regione_merge")

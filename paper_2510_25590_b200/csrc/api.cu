@@ -1,8 +1,6 @@
 // Host-only entry points of libregione: version, status names, the AVDCache
-// criterion (a scalar recurrence evaluated on the host), and the dispatcher of
-// the region attention.
-#include <cstdlib>
-#include <cstring>
+// criterion (a scalar recurrence evaluated on the host), and the argument checks
+// and entry points of the region attention.
 
 #include "common.cuh"
 
@@ -20,7 +18,7 @@ int launch_region_attention_tc(const uint16_t*, const uint16_t*, const uint16_t*
 
 using namespace regione;
 
-extern "C" int regione_version(void) { return 100; }
+extern "C" int regione_version(void) { return 200; }
 
 extern "C" const char* regione_status_string(int status) {
     switch (status) {
@@ -49,9 +47,24 @@ extern "C" int regione_avd_step(double* running_product, double dt, double gamma
     return REGIONE_OK;
 }
 
-static bool use_simt() {
-    const char* e = std::getenv("REGIONE_ATTENTION_IMPL");
-    return e != nullptr && std::strcmp(e, "simt") == 0;
+// Argument checks shared by every region-attention entry point.
+int regione::check_attention_args(const void* q, const void* k_fresh, const void* v_fresh,
+                                  const void* k_cache, const void* v_cache, const void* n_q,
+                                  const void* n_fresh, const void* n_cache, int B, int Nq_cap,
+                                  int Nf_cap, int Nc_cap, int H, int D, const void* out,
+                                  bool* nothing_to_do) {
+    *nothing_to_do = false;
+    if (!q || !out || !n_q || !n_fresh || !n_cache) return REGIONE_INVALID_ARG;
+    if (B < 0 || Nq_cap < 0 || Nf_cap < 0 || Nc_cap < 0 || H < 1) return REGIONE_INVALID_ARG;
+    if (Nf_cap > 0 && (!k_fresh || !v_fresh)) return REGIONE_INVALID_ARG;
+    if (Nc_cap > 0 && (!k_cache || !v_cache)) return REGIONE_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_fresh) || !aligned16(v_fresh) ||
+        !aligned16(k_cache) || !aligned16(v_cache))
+        return REGIONE_INVALID_ARG;
+    if (D != 64 && D != 128) return REGIONE_UNSUPPORTED;
+    if (B > 65535 || H > 65535) return REGIONE_UNSUPPORTED;
+    *nothing_to_do = (B == 0 || Nq_cap == 0);
+    return REGIONE_OK;
 }
 
 extern "C" size_t regione_region_attention_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap,
@@ -69,24 +82,11 @@ static int region_attention_impl(const regione_bf16* q, const regione_bf16* k_fr
                                  regione_bf16* out, const int32_t* out_rows, int out_cap,
                                  void* workspace, size_t workspace_bytes, int32_t* dev_status,
                                  void* stream) {
-    if (!q || !out || !n_q || !n_fresh || !n_cache) return REGIONE_INVALID_ARG;
-    if (B < 0 || Nq_cap < 0 || Nf_cap < 0 || Nc_cap < 0 || H < 1) return REGIONE_INVALID_ARG;
-    if (Nf_cap > 0 && (!k_fresh || !v_fresh)) return REGIONE_INVALID_ARG;
-    if (Nc_cap > 0 && (!k_cache || !v_cache)) return REGIONE_INVALID_ARG;
-    if (!aligned16(q) || !aligned16(out) || !aligned16(k_fresh) || !aligned16(v_fresh) ||
-        !aligned16(k_cache) || !aligned16(v_cache))
-        return REGIONE_INVALID_ARG;
-    if (D != 64 && D != 128) return REGIONE_UNSUPPORTED;
-    if (B > 65535 || H > 65535) return REGIONE_UNSUPPORTED;
-    if (B == 0 || Nq_cap == 0) return REGIONE_OK;
+    bool nothing = false;
+    const int rc = check_attention_args(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
+                                        B, Nq_cap, Nf_cap, Nc_cap, H, D, out, &nothing);
+    if (rc != REGIONE_OK || nothing) return rc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
-    cudaStream_t st = (cudaStream_t)stream;
-    if (use_simt()) {
-        if (out_rows != nullptr) return REGIONE_UNSUPPORTED;   // the cross-check path writes dense rows
-        return launch_region_attention_simt(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh,
-                                            n_cache, B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out,
-                                            dev_status, st);
-    }
     const size_t need = region_attention_tc_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D);
     if (need > 0) {
         if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return REGIONE_INVALID_ARG;
@@ -94,7 +94,7 @@ static int region_attention_impl(const regione_bf16* q, const regione_bf16* k_fr
     }
     return launch_region_attention_tc(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
                                       B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, out_rows, out_cap,
-                                      workspace, workspace_bytes, dev_status, st);
+                                      workspace, workspace_bytes, dev_status, (cudaStream_t)stream);
 }
 
 extern "C" int regione_region_attention(const regione_bf16* q, const regione_bf16* k_fresh,
@@ -119,4 +119,21 @@ extern "C" int regione_region_attention_scatter(
     return region_attention_impl(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, B,
                                  Nq_cap, Nf_cap, Nc_cap, H, D, softmax_scale, out_full, out_rows,
                                  out_rows_cap, workspace, workspace_bytes, dev_status, stream);
+}
+
+// The CUDA-core kernel, reachable only through this symbol: an independent arithmetic path on the
+// device that the tests compare the tensor-core kernel with.  Never called by the library itself.
+extern "C" int regione_crosscheck_region_attention(
+    const regione_bf16* q, const regione_bf16* k_fresh, const regione_bf16* v_fresh,
+    const regione_bf16* k_cache, const regione_bf16* v_cache, const int32_t* n_q,
+    const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap, int Nf_cap, int Nc_cap, int H,
+    int D, float softmax_scale, regione_bf16* out, int32_t* dev_status, void* stream) {
+    bool nothing = false;
+    const int rc = check_attention_args(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
+                                        B, Nq_cap, Nf_cap, Nc_cap, H, D, out, &nothing);
+    if (rc != REGIONE_OK || nothing) return rc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    return launch_region_attention_simt(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
+                                        B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, dev_status,
+                                        (cudaStream_t)stream);
 }

@@ -1,8 +1,8 @@
 // Plain CUDA-core region attention: one warp per (request, head, query row),
 // online softmax over the fresh rows and then the cached rows.  It exists to
 // cross-check the tensor-core kernel on the device (same inputs, independent
-// arithmetic path) and is selected with REGIONE_ATTENTION_IMPL=simt; it is
-// far from the tensor-core roofline and is never the default.
+// arithmetic path) and is reachable only through regione_crosscheck_region_attention; it is
+// far from the tensor-core roofline and no product entry point calls it.
 // (Sec. 4 "Region-Aware Generation", the attention equation.)
 #include "common.cuh"
 

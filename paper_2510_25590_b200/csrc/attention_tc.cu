@@ -67,7 +67,7 @@ constexpr int kBN = 128;                 // key rows per shared-memory tile
 constexpr int kBH = 64;                  // key rows per P chunk (half a tile)
 constexpr int kPolyEvery = 4;             // one pair in kPolyEvery computes one of its two exponentials on the FMA pipe
 constexpr int kHalfBytes = 128 * 64 * 2; // one 128-row x 64-column bf16 box (128-byte rows)
-constexpr long long kTimeoutCycles = 4000000000LL;
+constexpr long long kTimeoutCycles = 4000000000LL;   // default bound of every wait (about 2 s)
 
 template <int D>
 struct AttnCfg {
@@ -123,6 +123,7 @@ struct AttnParams {
     float* part_o;       // [B, H, P_cap, max_slots, 256, D] unnormalised outputs
     float2* part_ml;     // [B, H, P_cap, max_slots, 256]    (running max in the exp2 domain, sum)
     CutItem* cut;        // [grid] the item that the start of each share cuts, for the merge kernel
+    long long timeout_cycles;   // bound of every barrier wait, in SM clock cycles
 };
 
 
@@ -291,14 +292,17 @@ __device__ __forceinline__ Segment segment_ticks(const AttnParams& p, const Plan
     return sg;
 }
 
+// Bounded wait on phase `parity` of an mbarrier: true when the phase completed, false when another
+// role has already given up or `limit` cycles have passed (then the abort flag is raised and
+// REGIONE_DEV_TIMEOUT recorded; the caller leaves its loop, nothing traps).
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                         int32_t* dev_status) {
+                                         int32_t* dev_status, long long limit) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kTimeoutCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             record_status(dev_status, REGIONE_DEV_TIMEOUT);
             return false;
@@ -464,7 +468,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 const int stage = i % n_stages, use = i / n_stages;
                 if (use > 0)
                     ok = wait_bar(ptx::smem_addr(&ctrl->kv_empty[stage]), (use - 1) & 1, abort_flag,
-                                  p.dev_status);
+                                  p.dev_status, p.timeout_cycles);
                 if (!ok) break;
                 bool cached; int row0, valid;
                 tile_seg(j, cached, row0, valid);
@@ -511,11 +515,11 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                                 ptx::smem_desc_join(b0 + ((kk * 2048) >> 4), hi_k), idesc_pv,
                                 (accumulate || kk > 0) ? 1u : 0u);
             };
-            bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status);
+            bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status, p.timeout_cycles);
             if (ok) {
                 const int ik0 = 2 * role_tile(t, 0), sk0 = ik0 % n_stages;
                 ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk0]), (ik0 / n_stages) & 1, abort_flag,
-                              p.dev_status);
+                              p.dev_status, p.timeout_cycles);
                 if (ok) {
                     ptx::tc_fence_after_sync();
                     if (ptx::elect_one()) {
@@ -534,10 +538,10 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 const bool more = (j + 1 < n_my);
                 const int chunks = tile_chunks(jl);
                 ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / n_stages) & 1, abort_flag,
-                              p.dev_status);
+                              p.dev_status, p.timeout_cycles);
                 if (ok)
                     ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][0]), j & 1, abort_flag,
-                                  p.dev_status);
+                                  p.dev_status, p.timeout_cycles);
                 if (!ok) break;
                 if (chunks == 2) {
                     ptx::tc_fence_after_sync();
@@ -546,10 +550,10 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 }
                 if (more)
                     ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / n_stages) & 1, abort_flag,
-                                  p.dev_status);
+                                  p.dev_status, p.timeout_cycles);
                 if (ok && chunks == 2) {
                     ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][1]), nb & 1, abort_flag,
-                                  p.dev_status);
+                                  p.dev_status, p.timeout_cycles);
                     ++nb;
                 }
                 if (!ok) break;
@@ -584,7 +588,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             bool cached; int row0, valid;
             tile_seg(role_tile(t, j), cached, row0, valid);
             const int chunks = valid > kBH ? 2 : 1;
-            ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status);
+            ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status, p.timeout_cycles);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             // (P_t V_{j-1} has completed here: S_t(j) was issued after it by the same thread and
@@ -630,7 +634,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             // maxima and products fall into the gap.
             if (lanes == 2 && (t == 1 || j > 0)) {
                 ok = wait_bar(ptx::smem_addr(&ctrl->turn[t]), (j - 1 + t) & 1, abort_flag,
-                              p.dev_status);
+                              p.dev_status, p.timeout_cycles);
                 if (!ok) break;
             }
             // first chunk of probabilities (keys 0..63 of the tile)
@@ -642,7 +646,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
                 const int iv = 2 * role_tile(t, j) + 1, sv = iv % n_stages;
                 ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / n_stages) & 1, abort_flag,
-                              p.dev_status);
+                              p.dev_status, p.timeout_cycles);
                 if (!ok) break;
                 if (row >= valid) {
                     uint8_t* vrow = ring_gen + sv * kTileBytes + row * 128;
@@ -680,7 +684,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         if (live && direct)
             dst_row = p.out_rows != nullptr ? p.out_rows[(size_t)b * p.Nq_cap + wrow0 + lane] : wrow0 + lane;
         if (n_tiles > 0 && ok) {
-            ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status);
+            ok = wait_bar(ptx::smem_addr(&ctrl->o_final[t]), 0, abort_flag, p.dev_status, p.timeout_cycles);
             if (ok) ptx::tc_fence_after_sync();
         }
         // lone query tile: role 1 leaves its (max, sum) in shared memory (its accumulator stays in
@@ -692,8 +696,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->half_done));
         } else if (split && ok) {
-            ok = wait_bar(ptx::smem_addr(&ctrl->half_done), 0, abort_flag, p.dev_status);
-            if (ok) ok = wait_bar(ptx::smem_addr(&ctrl->o_final[1]), 0, abort_flag, p.dev_status);
+            ok = wait_bar(ptx::smem_addr(&ctrl->half_done), 0, abort_flag, p.dev_status, p.timeout_cycles);
+            if (ok) ok = wait_bar(ptx::smem_addr(&ctrl->o_final[1]), 0, abort_flag, p.dev_status, p.timeout_cycles);
             if (ok) {
                 ptx::tc_fence_after_sync();
                 const float2 other = half_ml[row];
@@ -952,17 +956,53 @@ region_attention_combine_kernel(const AttnParams p) {
         *reinterpret_cast<uint32_t*>(orow) = packed[0];
 }
 
+// Self-test of the bounded wait: one thread waits, through the same wait_bar the attention
+// kernel's roles use, on an mbarrier that nobody ever arrives on.  No copy and no tensor-core
+// operation is in flight, so giving up is all that happens: the wait must return false after
+// `limit` cycles with REGIONE_DEV_TIMEOUT recorded, and the kernel ends normally.
+// out[0] = 1 if the wait reported a completed phase (it must not), out[1] = cycles spent waiting.
+__global__ void bounded_wait_selftest_kernel(long long limit, int32_t* dev_status, long long* out) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        ptx::mbar_init(ptx::smem_addr(&bar), 1);
+        ptx::fence_barrier_init();
+        const long long t0 = clock64();
+        const bool done = wait_bar(ptx::smem_addr(&bar), 0, &abort_flag, dev_status, limit);
+        const long long spent = clock64() - t0;
+        if (out != nullptr) {
+            out[0] = done ? 1 : 0;
+            out[1] = spent;
+            out[2] = abort_flag;
+        }
+        ptx::mbar_inval(ptx::smem_addr(&bar));
+    }
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 
+constexpr int kMaxDevices = 64;
+
+// Ordinal of the current device, or -1 (no device / an ordinal beyond the per-device caches).
+static int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
+// SM count of the current device (cached per device; 148 when it cannot be read).
 static int sm_count() {
-    static int n = 0;
+    static int cached[kMaxDevices] = {};
+    const int dev = current_device();
+    if (dev < 0) return 148;
+    int n = __atomic_load_n(&cached[dev], __ATOMIC_ACQUIRE);
     if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            n = v;
-        else
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
             return 148;
+        n = v;
+        __atomic_store_n(&cached[dev], n, __ATOMIC_RELEASE);
     }
     return n;
 }
@@ -1032,13 +1072,16 @@ size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, 
 template <int D>
 static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, cudaStream_t st) {
     using Cfg = AttnCfg<D>;
-    static bool configured = false;
-    if (!configured) {
+    // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+    static int configured[kMaxDevices] = {};
+    const int dev = current_device();
+    if (dev < 0) return REGIONE_CUDA_ERROR;
+    if (!__atomic_load_n(&configured[dev], __ATOMIC_ACQUIRE)) {
         if (cudaFuncSetAttribute(region_attention_tc_kernel<D>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg::kSmemBytes) != cudaSuccess)
             return REGIONE_CUDA_ERROR;
-        configured = true;
+        __atomic_store_n(&configured[dev], 1, __ATOMIC_RELEASE);
     }
     if (launch_overlapped(region_attention_tc_kernel<D>, dim3(grid), dim3(kAttnThreads),
                           Cfg::kSmemBytes, st, maps[0], maps[1], maps[2], maps[3], maps[4],
@@ -1087,6 +1130,7 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
     prm.out = out; prm.dev_status = dev_status;
     prm.out_rows = out_rows;
     prm.out_cap = out_rows != nullptr ? out_cap : Nq_cap;
+    prm.timeout_cycles = kTimeoutCycles;
     const size_t rows = slot_rows(lp, B, H);
     prm.part_o = reinterpret_cast<float*>(workspace);
     uint8_t* const ws = reinterpret_cast<uint8_t*>(workspace);
@@ -1104,15 +1148,14 @@ constexpr size_t kStaticScratchBytes = (size_t)64 << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 namespace {
-constexpr int kMaxDevices = 64;
 void* g_static_scratch_addr[kMaxDevices] = {};      // device address of the array, per device
 }  // namespace
 
 // Device address of g_static_scratch on the current device (in host code the symbol itself is
 // only a stand-in and must never be handed to a kernel).  Resolved on the first call per device.
 static int static_scratch_address(void** out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return REGIONE_CUDA_ERROR;
+    const int dev = current_device();
+    if (dev < 0) return REGIONE_CUDA_ERROR;
     void* addr = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
     if (addr == nullptr) {
         if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || addr == nullptr) {
@@ -1127,22 +1170,25 @@ static int static_scratch_address(void** out) {
 
 }  // namespace regione
 
+extern "C" int regione_selftest_bounded_wait(long long limit_cycles, int32_t* dev_status,
+                                             long long* out, void* stream) {
+    using namespace regione;
+    // the limit is capped well below the attention kernel's own so that the self-test stays short
+    if (limit_cycles < 1 || limit_cycles > 100000000LL) return REGIONE_INVALID_ARG;
+    bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_cycles, dev_status, out);
+    return launch_status(cudaGetLastError());
+}
+
 extern "C" int regione_region_attention_static(
     const regione_bf16* q, const regione_bf16* k_fresh, const regione_bf16* v_fresh,
     const regione_bf16* k_cache, const regione_bf16* v_cache, const int32_t* n_q,
     const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap, int Nf_cap, int Nc_cap, int H,
     int D, float softmax_scale, regione_bf16* out, int32_t* dev_status, void* stream) {
     using namespace regione;
-    if (!q || !out || !n_q || !n_fresh || !n_cache) return REGIONE_INVALID_ARG;
-    if (B < 0 || Nq_cap < 0 || Nf_cap < 0 || Nc_cap < 0 || H < 1) return REGIONE_INVALID_ARG;
-    if (Nf_cap > 0 && (!k_fresh || !v_fresh)) return REGIONE_INVALID_ARG;
-    if (Nc_cap > 0 && (!k_cache || !v_cache)) return REGIONE_INVALID_ARG;
-    if (!aligned16(q) || !aligned16(out) || !aligned16(k_fresh) || !aligned16(v_fresh) ||
-        !aligned16(k_cache) || !aligned16(v_cache))
-        return REGIONE_INVALID_ARG;
-    if (D != 64 && D != 128) return REGIONE_UNSUPPORTED;
-    if (B > 65535 || H > 65535) return REGIONE_UNSUPPORTED;
-    if (B == 0 || Nq_cap == 0) return REGIONE_OK;
+    bool nothing = false;
+    const int args_rc = check_attention_args(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh,
+                                             n_cache, B, Nq_cap, Nf_cap, Nc_cap, H, D, out, &nothing);
+    if (args_rc != REGIONE_OK || nothing) return args_rc;
     // the partials of this shape must fit the fixed array: refuse, never truncate
     const size_t need = region_attention_tc_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D);
     if (need > kStaticScratchBytes) return REGIONE_WORKSPACE_TOO_SMALL;

@@ -74,6 +74,20 @@ inline cudaError_t launch_overlapped(void (*kernel)(Params...), dim3 grid, dim3 
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Per-request scalars (sampler time, step length, decay product) reach a kernel by value, a chunk
+// of requests per launch: the host arrays of the C ABI never have to be copied to device memory.
+constexpr int kReqChunk = 128;
+struct PerRequestF {
+    float v[kReqChunk];
+};
+
+// Host-side argument checks shared by every region-attention entry point (defined in api.cu).
+// Returns REGIONE_OK when the call may proceed; *nothing_to_do is set for B == 0 or Nq_cap == 0.
+int check_attention_args(const void* q, const void* k_fresh, const void* v_fresh, const void* k_cache,
+                         const void* v_cache, const void* n_q, const void* n_fresh, const void* n_cache,
+                         int B, int Nq_cap, int Nf_cap, int Nc_cap, int H, int D, const void* out,
+                         bool* nothing_to_do);
+
 inline int launch_status(cudaError_t e) { return e == cudaSuccess ? REGIONE_OK : REGIONE_CUDA_ERROR; }
 
 }  // namespace regione

@@ -1,6 +1,7 @@
 // Fitting the timestep-aware decay correction gamma_t of the Adaptive Velocity Decay Cache
-// (Sec. 4, decay-factor equation: ||v_{t_i}|| / ||v_{t_{i+1}}|| = (1 - dt_i) * gamma_{t_i}; the
-// paper obtains gamma "by fitting on a randomly sampled dataset").  Given the velocities of S
+// (Sec. 4 "Adaptive Velocity Decay Cache", decay-factor equation:
+// ||v_{t_i}|| / ||v_{t_{i+1}}|| = (1 - dt_i) * gamma_{t_i}; the paper fits gamma on sampled data and
+// does not say how).  Given the velocities of S
 // sampled trajectories at T+1 consecutive steps, gamma_i is the mean over the samples of the norm
 // ratio divided by the solver factor (1 - dt_i).
 //
@@ -15,6 +16,8 @@ constexpr int kNormThreads = 256;
 // norms[s, i] = || v[s, i, :] ||_2
 __global__ void __launch_bounds__(kNormThreads)
 velocity_norm_kernel(const uint4* __restrict__ v, long long chunks, float* __restrict__ norms) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const long long row = blockIdx.x;
     const uint4* p = v + row * chunks;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -54,6 +57,8 @@ velocity_norm_kernel(const uint4* __restrict__ v, long long chunks, float* __res
 // order the sampler takes them reversed: index i+1 is the earlier (noisier) step, as in the paper.
 __global__ void gamma_kernel(const float* __restrict__ norms, const float* __restrict__ dt, int S,
                              int T1, float* __restrict__ gamma) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= T1 - 1) return;
     float sum = 0.f;
@@ -75,8 +80,9 @@ extern "C" int regione_gamma_fit(const regione_bf16* v, int S, int T1, int64_t n
     if (!aligned16(v)) return REGIONE_INVALID_ARG;
     if ((n & 7) != 0 || (int64_t)S * T1 > 0x7fffffffLL) return REGIONE_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
-    velocity_norm_kernel<<<(unsigned)(S * T1), kNormThreads, 0, st>>>((const uint4*)v, n / 8, norms);
-    if (cudaGetLastError() != cudaSuccess) return REGIONE_CUDA_ERROR;
-    gamma_kernel<<<(T1 - 1 + 127) / 128, 128, 0, st>>>(norms, dt, S, T1, gamma);
-    return launch_status(cudaGetLastError());
+    if (launch_overlapped(velocity_norm_kernel, dim3((unsigned)(S * T1)), dim3(kNormThreads), 0, st,
+                          (const uint4*)v, (long long)(n / 8), norms) != cudaSuccess)
+        return REGIONE_CUDA_ERROR;
+    return launch_status(launch_overlapped(gamma_kernel, dim3((T1 - 1 + 127) / 128), dim3(128), 0, st,
+                                           (const float*)norms, dt, S, T1, gamma));
 }

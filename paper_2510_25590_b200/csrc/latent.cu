@@ -22,12 +22,13 @@ __device__ __forceinline__ uint4 axpy8(uint4 x, uint4 v, float a) {   // x + a *
 
 // x_e <- x_e - dt * (scale * v_in); optionally v_cache_out <- v_in.  One thread = 8 channels.
 __global__ void __launch_bounds__(kLatThreads)
-velocity_decay_kernel(const uint4* __restrict__ v_in, float neg_dt_scale, uint4* __restrict__ x_e,
-                      uint4* __restrict__ v_cache_out, const int32_t* __restrict__ n_edit,
-                      int Ne_cap, int cpr, int32_t* dev_status) {
+velocity_decay_kernel(const uint4* __restrict__ v_in, const PerRequestF neg_dt_scale_v, int b0,
+                      uint4* __restrict__ x_e, uint4* __restrict__ v_cache_out,
+                      const int32_t* __restrict__ n_edit, int Ne_cap, int cpr, int32_t* dev_status) {
     grid_dependency_wait();
     grid_launch_dependents();
-    const int b = blockIdx.y;
+    const int b = b0 + blockIdx.y;                       // requests b0 .. b0 + gridDim.y of the batch
+    const float neg_dt_scale = neg_dt_scale_v.v[blockIdx.y];
     int ne = n_edit[b];
     if (ne < 0 || ne > Ne_cap) {
         if (threadIdx.x == 0 && blockIdx.x == 0) record_status(dev_status, REGIONE_DEV_BOUNDS);
@@ -50,11 +51,13 @@ constexpr int kMergeUnroll = 4;
 
 __global__ void __launch_bounds__(kLatThreads)
 merge_kernel(const uint4* x_full, const uint4* __restrict__ v_last,
-             const uint4* __restrict__ x_e, const int32_t* __restrict__ slot, float neg_dt, int N,
-             int Ne_cap, int cpr, uint4* x_out, int32_t* dev_status) {
+             const uint4* __restrict__ x_e, const int32_t* __restrict__ slot,
+             const PerRequestF neg_dt_v, int b0, int N, int Ne_cap, int cpr, uint4* x_out,
+             int32_t* dev_status) {
     grid_dependency_wait();
     grid_launch_dependents();
-    const int b = blockIdx.y;
+    const int b = b0 + blockIdx.y;
+    const float neg_dt = neg_dt_v.v[blockIdx.y];
     const unsigned total = (unsigned)N * (unsigned)cpr;
     const unsigned base = blockIdx.x * (unsigned)(kLatThreads * kMergeUnroll) + threadIdx.x;
     const size_t req = (size_t)b * N * cpr;
@@ -98,29 +101,35 @@ merge_kernel(const uint4* x_full, const uint4* __restrict__ v_last,
 
 using namespace regione;
 
-extern "C" int regione_velocity_decay(const regione_bf16* v_in, float scale, float dt,
+extern "C" int regione_velocity_decay(const regione_bf16* v_in, const float* scale, const float* dt,
                                       regione_bf16* x_e, regione_bf16* v_cache_out,
                                       const int32_t* n_edit, int B, int Ne_cap, int C,
                                       int32_t* dev_status, void* stream) {
-    if (!v_in || !x_e || !n_edit) return REGIONE_INVALID_ARG;
+    if (!v_in || !x_e || !n_edit || !scale || !dt) return REGIONE_INVALID_ARG;
     if (B < 0 || Ne_cap < 0 || C < 1) return REGIONE_INVALID_ARG;
     if (!aligned16(v_in) || !aligned16(x_e) || !aligned16(v_cache_out)) return REGIONE_INVALID_ARG;
     if ((C & 7) != 0 || B > 65535) return REGIONE_UNSUPPORTED;
     const long long cpr = C / 8, total = (long long)Ne_cap * cpr;
     if (total + kLatThreads >= 0x7fffffffLL) return REGIONE_UNSUPPORTED;
     if (B == 0 || Ne_cap == 0) return REGIONE_OK;
-    dim3 grid((unsigned)((total + kLatThreads - 1) / kLatThreads), B);
-    // scale * v is formed first in fp32, then the Euler step: x - dt * (scale * v)
-    return launch_status(launch_overlapped(
-        velocity_decay_kernel, grid, dim3(kLatThreads), 0, (cudaStream_t)stream, (const uint4*)v_in,
-        -(dt * scale), (uint4*)x_e, (uint4*)v_cache_out, n_edit, Ne_cap, (int)cpr, dev_status));
+    cudaError_t e = cudaSuccess;
+    for (int b0 = 0; b0 < B && e == cudaSuccess; b0 += kReqChunk) {
+        const int nb = B - b0 < kReqChunk ? B - b0 : kReqChunk;
+        PerRequestF a;                       // x - (dt * scale) * v, the product formed in fp32 first
+        for (int i = 0; i < nb; ++i) a.v[i] = -(dt[b0 + i] * scale[b0 + i]);
+        dim3 grid((unsigned)((total + kLatThreads - 1) / kLatThreads), nb);
+        e = launch_overlapped(velocity_decay_kernel, grid, dim3(kLatThreads), 0, (cudaStream_t)stream,
+                              (const uint4*)v_in, a, b0, (uint4*)x_e, (uint4*)v_cache_out, n_edit,
+                              Ne_cap, (int)cpr, dev_status);
+    }
+    return launch_status(e);
 }
 
 extern "C" int regione_merge(const regione_bf16* x_full, const regione_bf16* v_last_full,
-                             const regione_bf16* x_e, const int32_t* slot, float dt_unedited, int B,
+                             const regione_bf16* x_e, const int32_t* slot, const float* dt_unedited, int B,
                              int N, int Ne_cap, int C, regione_bf16* x_out, int32_t* dev_status,
                              void* stream) {
-    if (!x_full || !v_last_full || !slot || !x_out) return REGIONE_INVALID_ARG;
+    if (!x_full || !v_last_full || !slot || !x_out || !dt_unedited) return REGIONE_INVALID_ARG;
     if (B < 0 || N < 1 || Ne_cap < 0 || C < 1) return REGIONE_INVALID_ARG;
     if (Ne_cap > 0 && !x_e) return REGIONE_INVALID_ARG;
     if (!aligned16(x_full) || !aligned16(v_last_full) || !aligned16(x_e) || !aligned16(x_out))
@@ -130,9 +139,15 @@ extern "C" int regione_merge(const regione_bf16* x_full, const regione_bf16* v_l
     if (total + kLatThreads >= 0x7fffffffLL) return REGIONE_UNSUPPORTED;
     if (B == 0) return REGIONE_OK;
     const long long per_block = (long long)kLatThreads * kMergeUnroll;
-    dim3 grid((unsigned)((total + per_block - 1) / per_block), B);
-    return launch_status(launch_overlapped(
-        merge_kernel, grid, dim3(kLatThreads), 0, (cudaStream_t)stream, (const uint4*)x_full,
-        (const uint4*)v_last_full, (const uint4*)x_e, slot, -dt_unedited, N, Ne_cap, (int)cpr,
-        (uint4*)x_out, dev_status));
+    cudaError_t e = cudaSuccess;
+    for (int b0 = 0; b0 < B && e == cudaSuccess; b0 += kReqChunk) {
+        const int nb = B - b0 < kReqChunk ? B - b0 : kReqChunk;
+        PerRequestF a;
+        for (int i = 0; i < nb; ++i) a.v[i] = -dt_unedited[b0 + i];
+        dim3 grid((unsigned)((total + per_block - 1) / per_block), nb);
+        e = launch_overlapped(merge_kernel, grid, dim3(kLatThreads), 0, (cudaStream_t)stream,
+                              (const uint4*)x_full, (const uint4*)v_last_full, (const uint4*)x_e, slot, a,
+                              b0, N, Ne_cap, (int)cpr, (uint4*)x_out, dev_status);
+    }
+    return launch_status(e);
 }

@@ -126,8 +126,8 @@ __device__ __forceinline__ void accumulate_chunk(uint4 xv, uint4 vv, uint4 rv, f
 template <int L>
 __global__ void __launch_bounds__(kPartMaxThreads)
 partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ v,
-                 const uint16_t* __restrict__ ref, int N, int C, int share, float t, int metric,
-                 float threshold, uint8_t* __restrict__ mask, int32_t* __restrict__ edit_idx,
+                 const uint16_t* __restrict__ ref, int N, int C, int share, const PerRequestF tv,
+                 int b0, int metric, float threshold, uint8_t* __restrict__ mask, int32_t* __restrict__ edit_idx,
                  int32_t* __restrict__ keep_idx, int32_t* __restrict__ slot,
                  int32_t* __restrict__ n_edit, float* __restrict__ score, const RowLists rl,
                  int32_t* dev_status) {
@@ -143,7 +143,8 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = cluster.block_rank();
     const int csize = cluster.num_blocks();
-    const int b = blockIdx.y;
+    const int b = b0 + blockIdx.y;               // this launch covers requests b0 .. b0 + gridDim.y
+    const float t = tv.v[blockIdx.y];            // the request's own sampler time
     const int start = rank * share;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int TPI = 32 / L;                 // tokens per sub-iteration
@@ -285,6 +286,8 @@ mask_open_close_kernel(const uint8_t* __restrict__ mask_in, int rows, int cols,
                        uint8_t* __restrict__ mask_out, int32_t* __restrict__ edit_idx,
                        int32_t* __restrict__ keep_idx, int32_t* __restrict__ slot,
                        int32_t* __restrict__ n_edit) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     __shared__ uint8_t bufA[kMorphMaxTokens];
     __shared__ uint8_t bufB[kMorphMaxTokens];
     __shared__ uint32_t bits[kMorphMaxTokens / 32];
@@ -361,7 +364,8 @@ using namespace regione;
 template <int L>
 static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st,
                                     const uint16_t* x_t, const uint16_t* v, const uint16_t* ref,
-                                    int N, int C, float t, int metric, float thr, uint8_t* mask,
+                                    int N, int C, const PerRequestF& tv, int b0, int metric,
+                                    float thr, uint8_t* mask,
                                     int32_t* edit_idx, int32_t* keep_idx, int32_t* slot,
                                     int32_t* n_edit, float* score, const RowLists& rl,
                                     int32_t* dev_status) {
@@ -383,17 +387,17 @@ static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, partition_kernel<L>, x_t, v, ref, N, C, share, t, metric, thr,
-                              mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status);
+    return cudaLaunchKernelEx(&cfg, partition_kernel<L>, x_t, v, ref, N, C, share, tv, b0, metric,
+                              thr, mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status);
 }
 
 static int partition_impl(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
-                          int B, int N, int C, float t, int metric, float threshold, uint8_t* mask,
+                          int B, int N, int C, const float* t, int metric, float threshold, uint8_t* mask,
                           int32_t* edit_idx, int32_t* keep_idx, int32_t* slot, int32_t* n_edit,
                           float* score, const RowLists& rl, int32_t* dev_status, void* stream) {
     if (!x_t || !v || !ref || !mask || !edit_idx || !keep_idx || !slot || !n_edit)
         return REGIONE_INVALID_ARG;
-    if (B < 0 || N < 1 || C < 1) return REGIONE_INVALID_ARG;
+    if (B < 0 || N < 1 || C < 1 || (B > 0 && !t)) return REGIONE_INVALID_ARG;
     if (!aligned16(x_t) || !aligned16(v) || !aligned16(ref)) return REGIONE_INVALID_ARG;
     if (metric != REGIONE_METRIC_COSINE && metric != REGIONE_METRIC_L2) return REGIONE_INVALID_ARG;
     if ((C & 7) != 0 || C > 4096 || B > 65535) return REGIONE_UNSUPPORTED;
@@ -406,29 +410,37 @@ static int partition_impl(const regione_bf16* x_t, const regione_bf16* v, const 
     int L = 1;
     while (L < 32 && L * 8 < C) L <<= 1;
     cudaStream_t st = (cudaStream_t)stream;
-    cudaError_t e;
+    cudaError_t e = cudaSuccess;
+    // the per-request times travel by value, kReqChunk requests per launch
+    for (int b0 = 0; b0 < B && e == cudaSuccess; b0 += kReqChunk) {
+        const int nb = B - b0 < kReqChunk ? B - b0 : kReqChunk;
+        PerRequestF tv;
+        for (int i = 0; i < nb; ++i) tv.v[i] = t[b0 + i];
 #define REGIONE_PART_CASE(LL)                                                                   \
     case LL:                                                                                    \
-        e = launch_partition<LL>(csize, B, share, st, x_t, v, ref, N, C, t, metric, threshold,  \
-                                 mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status); \
+        e = launch_partition<LL>(csize, nb, share, st, x_t, v, ref, N, C, tv, b0, metric,       \
+                                 threshold, mask, edit_idx, keep_idx, slot, n_edit, score, rl,  \
+                                 dev_status);                                                   \
         break;
-    switch (L) {
-        REGIONE_PART_CASE(1)
-        REGIONE_PART_CASE(2)
-        REGIONE_PART_CASE(4)
-        REGIONE_PART_CASE(8)
-        REGIONE_PART_CASE(16)
-        default:
-            e = launch_partition<32>(csize, B, share, st, x_t, v, ref, N, C, t, metric, threshold,
-                                     mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status);
+        switch (L) {
+            REGIONE_PART_CASE(1)
+            REGIONE_PART_CASE(2)
+            REGIONE_PART_CASE(4)
+            REGIONE_PART_CASE(8)
+            REGIONE_PART_CASE(16)
+            default:
+                e = launch_partition<32>(csize, nb, share, st, x_t, v, ref, N, C, tv, b0, metric,
+                                         threshold, mask, edit_idx, keep_idx, slot, n_edit, score, rl,
+                                         dev_status);
+        }
     }
 #undef REGIONE_PART_CASE
     return launch_status(e);
 }
 
 extern "C" int regione_partition(const regione_bf16* x_t, const regione_bf16* v,
-                                 const regione_bf16* ref, int B, int N, int C, float t, int metric,
-                                 float threshold, uint8_t* mask, int32_t* edit_idx,
+                                 const regione_bf16* ref, int B, int N, int C, const float* t,
+                                 int metric, float threshold, uint8_t* mask, int32_t* edit_idx,
                                  int32_t* keep_idx, int32_t* slot, int32_t* n_edit, float* score,
                                  int32_t* dev_status, void* stream) {
     RowLists none = {};
@@ -437,7 +449,7 @@ extern "C" int regione_partition(const regione_bf16* x_t, const regione_bf16* v,
 }
 
 extern "C" int regione_partition_rows(const regione_bf16* x_t, const regione_bf16* v,
-                                      const regione_bf16* ref, int B, int N, int C, float t,
+                                      const regione_bf16* ref, int B, int N, int C, const float* t,
                                       int metric, float threshold, uint8_t* mask, int32_t* edit_idx,
                                       int32_t* keep_idx, int32_t* slot, int32_t* n_edit, float* score,
                                       int n_text, int n_ref, int membership, int32_t* query_rows,
@@ -458,15 +470,15 @@ extern "C" int regione_mask_open_close(const uint8_t* mask_in, int B, int rows, 
                                        uint8_t* mask_out, int32_t* edit_idx, int32_t* keep_idx,
                                        int32_t* slot, int32_t* n_edit, int32_t* dev_status,
                                        void* stream) {
-    (void)dev_status;
+    (void)dev_status;      // no count or index input exists that could be out of range on the device
     if (!mask_in || !mask_out || !edit_idx || !keep_idx || !slot || !n_edit)
         return REGIONE_INVALID_ARG;
     if (B < 0 || rows < 1 || cols < 1 || mask_in == mask_out) return REGIONE_INVALID_ARG;
     if ((int64_t)rows * cols > kMorphMaxTokens) return REGIONE_UNSUPPORTED;
     if (B == 0) return REGIONE_OK;
-    mask_open_close_kernel<<<B, kMorphThreads, 0, (cudaStream_t)stream>>>(
-        mask_in, rows, cols, mask_out, edit_idx, keep_idx, slot, n_edit);
-    return launch_status(cudaGetLastError());
+    return launch_status(launch_overlapped(mask_open_close_kernel, dim3(B), dim3(kMorphThreads), 0,
+                                           (cudaStream_t)stream, mask_in, rows, cols, mask_out,
+                                           edit_idx, keep_idx, slot, n_edit));
 }
 
 extern "C" int regione_region_rows(const int32_t* edit_idx, const int32_t* keep_idx,

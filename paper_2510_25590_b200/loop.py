@@ -87,6 +87,16 @@ class RegionELoop:
         self.dev_status = z(1, dt=i32)
         self.hook = None             # optional callable(event: str, k: int, tensors: dict)
 
+    @staticmethod
+    def _copy(dst, src, stream):
+        """Device-to-device copy ordered on the same stream as the library calls around it."""
+        import torch
+        if stream is None:
+            dst.copy_(src)
+        else:
+            with torch.cuda.stream(stream):
+                dst.copy_(src)
+
     def _emit(self, event, k, **tensors):
         if self.hook is not None:
             self.hook(event, k, tensors)
@@ -116,7 +126,7 @@ class RegionELoop:
                     in_run = False
                 v = model.full(x, t_cur, partitioned or k + 1 == cfg.partition_after)
                 tr.model_full_calls += 1
-                self.v_last_full.copy_(v)
+                self._copy(self.v_last_full, v, stream)
                 self._emit("euler_in", k, x=x, v=v, dt=dt)
                 b.velocity_decay(v, 1.0, dt, x, self.n_all, dev_status=st, stream=stream)
                 self._emit("euler_out", k, x=x)
@@ -135,7 +145,7 @@ class RegionELoop:
             if not partitioned:
                 raise binding.RegionEError("a region step was scheduled before the partition")
             if not in_run:
-                self.x_run_start.copy_(x)
+                self._copy(self.x_run_start, x, stream)
                 b.gather(x, self.edit_idx, self.n_edit, self.x_e, dev_status=st, stream=stream)
                 tr.launches += 1
                 in_run, t_run = True, t_cur

@@ -40,13 +40,19 @@ def test_missing_library_fails_loudly(tmp_path):
 def test_argument_validation_happens_on_the_host():
     lib = binding.load()
     null = None
-    assert lib.regione_partition(null, null, null, 1, 8, 16, 0.5, 0, 0.9, null, null, null, null, null,
+    t1 = (ctypes.c_float * 1)(0.5)
+    assert lib.regione_partition(null, null, null, 1, 8, 16, t1, 0, 0.9, null, null, null, null, null,
                                  null, null, null) == binding.INVALID_ARG
     fake = ctypes.c_void_p(4096)
-    assert lib.regione_partition(fake, fake, fake, 1, 8, 12, 0.5, 0, 0.9, fake, fake, fake, fake, fake,
+    assert lib.regione_partition(fake, fake, fake, 1, 8, 12, t1, 0, 0.9, fake, fake, fake, fake, fake,
                                  null, null, null) == binding.UNSUPPORTED         # C % 8 != 0
-    assert lib.regione_partition(fake, fake, fake, 1, 8, 16, 0.5, 7, 0.9, fake, fake, fake, fake, fake,
+    assert lib.regione_partition(fake, fake, fake, 1, 8, 16, t1, 7, 0.9, fake, fake, fake, fake, fake,
                                  null, null, null) == binding.INVALID_ARG         # unknown metric
+    assert lib.regione_partition(fake, fake, fake, 1, 8, 16, null, 0, 0.9, fake, fake, fake, fake, fake,
+                                 null, null, null) == binding.INVALID_ARG         # no per-request times
+    # one request may hold at most 2^20 tokens
+    assert lib.regione_partition(fake, fake, fake, 1, (1 << 20) + 1, 16, t1, 0, 0.9, fake, fake, fake, fake,
+                                 fake, null, null, null) == binding.UNSUPPORTED
     odd = ctypes.c_void_p(4100)
     assert lib.regione_gather(odd, fake, fake, 1, 4, 4, 4, 32, fake, null, null) == binding.INVALID_ARG
     assert lib.regione_gather(fake, fake, fake, 1, 4, 4, 4, 24, fake, null, null) == binding.UNSUPPORTED
@@ -57,10 +63,18 @@ def test_argument_validation_happens_on_the_host():
                                         0.0, fake, null, 0, null, null) == binding.UNSUPPORTED
     assert lib.regione_region_attention(fake, null, null, fake, fake, fake, fake, fake, 1, 8, 8, 8, 2, 64,
                                         0.0, fake, null, 0, null, null) == binding.INVALID_ARG
-    assert lib.regione_velocity_decay(fake, 1.0, 0.1, fake, null, fake, 1, 8, 10, null, null) \
+    assert lib.regione_velocity_decay(fake, t1, t1, fake, null, fake, 1, 8, 10, null, null) \
         == binding.UNSUPPORTED
-    assert lib.regione_merge(fake, fake, null, fake, 0.1, 1, 8, 4, 16, fake, null, null) \
+    assert lib.regione_velocity_decay(fake, null, t1, fake, null, fake, 1, 8, 16, null, null) \
         == binding.INVALID_ARG
+    assert lib.regione_merge(fake, fake, null, fake, t1, 1, 8, 4, 16, fake, null, null) \
+        == binding.INVALID_ARG
+    assert lib.regione_merge(fake, fake, fake, fake, null, 1, 8, 4, 16, fake, null, null) \
+        == binding.INVALID_ARG
+    assert lib.regione_crosscheck_region_attention(fake, fake, fake, fake, fake, fake, fake, fake, 1, 8, 8, 8,
+                                                   2, 96, 0.0, fake, null, null) == binding.UNSUPPORTED
+    assert lib.regione_selftest_bounded_wait(0, null, null, null) == binding.INVALID_ARG
+    assert lib.regione_selftest_bounded_wait(10 ** 9, null, null, null) == binding.INVALID_ARG
     assert lib.regione_mask_open_close(fake, 1, 200, 200, ctypes.c_void_p(8192), fake, fake, fake, fake,
                                        null, null) == binding.UNSUPPORTED
     assert lib.regione_region_attention_workspace(1, 128, 128, 128, 4, 96) == 0

@@ -28,8 +28,8 @@ class TorchStraightLine:
         return ((x_e.float() - tgt) / t).to(x_e.dtype)
 
 
-def _case(seed=5, B=2, grid=(24, 24), ratio=0.25):
-    wl = synth.scaled_workload(synth.WORKLOADS[1], grid=grid, batch=B)
+def _case(seed=5, B=2, grid=(24, 24), ratio=0.25, base=1):
+    wl = synth.scaled_workload(synth.WORKLOADS[base], grid=grid, batch=B)
     lat = synth.make_latents(wl, ratio, stream=seed)
     rng = np.random.default_rng(seed)
     ref = lat["ref"]
@@ -39,16 +39,25 @@ def _case(seed=5, B=2, grid=(24, 24), ratio=0.25):
     return wl, ref, m, target, noise
 
 
-@pytest.mark.parametrize("which,n_steps", [("alternating", 28), ("alternating", 10), ("paper", 28)])
-def test_loop_calls_match_oracle_step_by_step(which, n_steps):
+@pytest.mark.parametrize("which,n_steps,full_size", [("alternating", 28, False), ("alternating", 10, False),
+                                                     ("paper", 28, False), ("alternating", 28, True),
+                                                     ("paper", 28, True)])
+def test_loop_calls_match_oracle_step_by_step(which, n_steps, full_size):
+    """full_size: the Step1X-Edit-shaped loop at its own size (64 x 64 latent = 4096 tokens of 16 channels,
+    one request, two-ellipse mask of 20 %, per-token L2 threshold 0.1), 28 steps under either schedule."""
     import torch
-    wl, ref, m, target, noise = _case()
+    if full_size:
+        wl, ref, m, target, noise = _case(seed=4, B=1, grid=(64, 64), ratio=0.20, base=4)
+        metric_g, metric_o, thr = binding.METRIC_L2, orc.L2, 0.1
+    else:
+        wl, ref, m, target, noise = _case()
+        metric_g, metric_o, thr = binding.METRIC_COSINE, orc.COSINE, 0.9
     kinds, after = gloop.alternating_schedule() if which == "alternating" else gloop.paper_schedule()
     T = len(kinds)
     ts = [1.0 - k / T for k in range(T + 1)]
     kinds, ts = kinds[:n_steps], ts[:n_steps + 1]
     delta = 0.05 if which == "alternating" else 0.04
-    cfg = gloop.LoopConfig(kinds, after, ts, [1.0] * (T + 1), delta, binding.METRIC_COSINE, 0.9)
+    cfg = gloop.LoopConfig(kinds, after, ts, [1.0] * (T + 1), delta, metric_g, thr)
     B, N, C = noise.shape
     lp = gloop.RegionELoop(B, N, C, cfg)
     pending = {}
@@ -64,7 +73,7 @@ def test_loop_calls_match_oracle_step_by_step(which, n_steps):
             want = inp["x"] - np.float32(inp["dt"]).astype(np.float64) * inp["v"]
             assert_close(grab["x"], want, f"euler step {k}")
         elif name == "partition":
-            p = orc.partition(inp["x"], inp["v"], inp["ref"], np.float32(inp["t"]), orc.COSINE, np.float32(0.9))
+            p = orc.partition(inp["x"], inp["v"], inp["ref"], np.float32(inp["t"]), metric_o, np.float32(thr))
             assert np.array_equal(grab["mask"], p["mask"]) and np.array_equal(grab["slot"], p["slot"])
             assert np.array_equal(grab["n_edit"], p["n_edit"])
             assert np.array_equal(p["mask"].astype(bool), m)
@@ -86,7 +95,7 @@ def test_loop_calls_match_oracle_step_by_step(which, n_steps):
     assert {"euler", "partition", "decay", "merge"} <= set(checked)
 
     res = loop_oracle.run_loop(noise, ref, loop_oracle.StraightLineModel(target), kinds, after, ts,
-                               np.ones(T + 1), delta, orc.COSINE, 0.9)
+                               np.ones(T + 1), delta, metric_o, thr)
     assert [(k, kind, w) for k, kind, w, _ in trace.steps] == [(k, kind, w) for k, kind, w, _ in res["log"]]
     for (_, _, _, s_gpu), (_, _, _, s_orc) in zip(trace.steps, res["log"]):
         assert abs(s_gpu - s_orc) < 1e-12

@@ -226,3 +226,24 @@ def test_partition_with_row_lists_reports_lists_that_do_not_fit():
     torch.cuda.synchronize()
     assert int(st[0]) == binding.DEV_BOUNDS
     assert int(nq[0]) == 8 and int(nc[0]) == 8                       # clamped, nothing written past the end
+
+
+@pytest.mark.parametrize("B", [3, 130])
+def test_requests_at_their_own_sampler_times(B):
+    """Each request of a batch carries its own t (requests sitting at different sampler steps, or the
+    two guidance branches of one request sharing a mask): request b must equal the oracle run on that
+    request alone with t[b].  B = 130 crosses the 128-requests-per-launch chunk of the time array."""
+    wl = synth.scaled_workload(synth.WORKLOADS[5], grid=(20, 20), batch=B)
+    ts = [(22.0 - (b % 5)) / 28.0 for b in range(B)]
+    lats = [synth.make_latents(synth.scaled_workload(wl, batch=1), stream=b, t=ts[b]) for b in range(B)]
+    x_t, v, ref = (np.concatenate([l[k] for l in lats]) for k in ("x_t", "v", "ref"))
+    got = run_partition(x_t, v, ref, ts, orc.COSINE, wl.threshold)
+    for b in range(B):
+        want = orc.partition(x_t[b:b + 1], v[b:b + 1], ref[b:b + 1], np.float32(ts[b]), orc.COSINE, wl.threshold)
+        one = {k: a[b:b + 1] for k, a in got.items()}
+        check_against_oracle(one, want, wl.n_img)
+        assert np.array_equal(one["mask"][0], lats[b]["mask"][0])
+    # the same batch with every request at the first request's time decides some tokens differently
+    # (otherwise this test would not notice a kernel that ignores the per-request values)
+    same = run_partition(x_t, v, ref, ts[0], orc.COSINE, wl.threshold)
+    assert not np.array_equal(same["score"], got["score"])

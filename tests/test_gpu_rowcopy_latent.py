@@ -161,3 +161,40 @@ def test_gather_multi_matches_single_gathers():
         assert torch.equal(a, b_)
     with pytest.raises(binding.RegionEError):
         binding.gather_multi(srcs * 2, idx, n, many * 2)
+
+
+@pytest.mark.parametrize("B", [4, 131])
+def test_velocity_decay_and_merge_with_per_request_steps(B):
+    """Requests of one batch at different sampler steps: scale, dt and dt_unedited are arrays of B
+    values; request b must match the oracle called on that request alone with its own values."""
+    import torch
+    rng = np.random.default_rng(B)
+    cap, C, N = 90, 16, 160
+    v, x = _rand_bf16(rng, (B, cap, C)), _rand_bf16(rng, (B, cap, C))
+    n = rng.integers(1, cap + 1, B).astype(np.int32)
+    scale = (0.8 + 0.2 * rng.random(B)).astype(np.float32)
+    dt = ((1 + rng.integers(0, 4, B)) / 28.0).astype(np.float32)
+    dx = dev_bf16(x)
+    binding.velocity_decay(dev_bf16(v), scale, dt, dx, dev_i32(n))
+    got = host_f64(dx)
+    for b in range(B):
+        want, _ = orc.velocity_decay(v[b:b + 1], scale[b], dt[b], x[b:b + 1], n[b:b + 1])
+        assert np.all(np.abs(got[b] - want[0]) <= 2.0 ** -8 * np.abs(want[0]) + 1e-6), b
+    assert len(set(np.round(dt * scale, 6).tolist())) > 2          # the values really differ
+    # merge
+    xf, vf = _rand_bf16(rng, (B, N, C)), _rand_bf16(rng, (B, N, C))
+    slot = np.full((B, N), -1, np.int32)
+    for b in range(B):
+        ids = np.sort(rng.permutation(N)[:n[b]])
+        slot[b, ids] = np.arange(n[b])
+    dtu = ((2 + rng.integers(0, 6, B)) / 28.0).astype(np.float32)
+    out = torch.full((B, N, C), -3.0, dtype=torch.bfloat16, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    binding.merge(dev_bf16(xf), dev_bf16(vf), dev_bf16(x), dev_i32(slot), dtu, out, dev_status=st)
+    got = host_f64(out)
+    assert int(st[0]) == 0
+    for b in range(B):
+        want = orc.merge(xf[b:b + 1], vf[b:b + 1], x[b:b + 1], slot[b:b + 1], dtu[b])
+        assert np.all(np.abs(got[b] - want[0]) <= 2.0 ** -8 * np.abs(want[0]) + 1e-6), b
+    with pytest.raises(binding.RegionEError):
+        binding.merge(dev_bf16(xf), dev_bf16(vf), dev_bf16(x), dev_i32(slot), dtu[:2], out)

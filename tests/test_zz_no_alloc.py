@@ -3,9 +3,9 @@
 Some users of this library cannot allocate device memory at the call site (a server whose arena
 already owns all of HBM, a step loop that must avoid the device-wide stall of cudaMalloc), so the
 library carries a fixed scratch array for the split-KV partials.  This file checks, through the
-C ABI, that the variant gives the same result as the ordinary entry point, twice in a row with
-different inputs (the scratch keeps the first call's contents), and that an oversized shape is
-refused.  It is named to be collected last.
+C ABI, that the variant gives the same result as the ordinary entry point and as the fp64 oracle,
+twice in a row with different inputs (the scratch keeps the first call's contents), and that an
+oversized shape is refused.  It is named to be collected last.
 """
 import ctypes
 
@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 
 from gpu_util import assert_close, dev_bf16, dev_i32, host_f64
+from oracle import regione_oracle as orc
 from paper_2510_25590_b200 import binding, synth
 
 pytestmark = pytest.mark.gpu
@@ -31,8 +32,10 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
     assert ws_bytes > 0, "shape must use split-KV, otherwise no scratch is exercised"
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     n_q, n_f, n_c = dev_i32([nq, nq - 41]), dev_i32([nf, 17]), dev_i32([nc, nc - 333])
+    counts = (np.array([nq, nq - 41]), np.array([nf, 17]), np.array([nc, nc - 333]))
     for call, seed in enumerate((11, 12)):
-        q, kf, vf, kc, vc = (dev_bf16(a) for a in _case(seed, B, nq, nf, nc, H, D))
+        host = _case(seed, B, nq, nf, nc, H, D)
+        q, kf, vf, kc, vc = (dev_bf16(a) for a in host)
         want = torch.full(q.shape, -3.0, dtype=torch.bfloat16, device="cuda")
         got = torch.full(q.shape, -3.0, dtype=torch.bfloat16, device="cuda")
         st = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -44,6 +47,10 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
         assert np.array_equal(g[0, nq:], w[0, nq:]) and np.array_equal(g[1, nq - 41:], w[1, nq - 41:])
         assert_close(g[0, :nq], w[0, :nq], f"call {call}, request 0")
         assert_close(g[1, :nq - 41], w[1, :nq - 41], f"call {call}, request 1")
+        # and against the fp64 oracle directly, every live row
+        ref = orc.region_attention(*host, *counts)
+        assert_close(g[0, :nq], ref[0, :nq], f"call {call}, request 0 vs oracle")
+        assert_close(g[1, :nq - 41], ref[1, :nq - 41], f"call {call}, request 1 vs oracle")
 
 
 def test_static_scratch_variant_refuses_shapes_beyond_its_array():
