@@ -361,8 +361,57 @@ def per_config_rows(torch, binding, synth, flush_l2, to_dev, peaks, steps=12):
                          step_tflops_equivalent=round(fl / st_us / 1e6, 1)))
         del step, dq, dk, dv
         torch.cuda.empty_cache()
+    rows.append(full_step_row(torch, binding, synth, flush_l2, to_dev, peaks))
     rows.append(loop_row(torch, binding, synth, to_dev))
     return rows
+
+
+def full_step_row(torch, binding, synth, flush_l2, to_dev, peaks, iters=10):
+    """The forced full step on the Qwen-Image-Edit-shaped layer (8448 joint rows, 24 heads x 128, the
+    cache keeps text + unedited + reference rows of the 25 % mask): plain joint attention followed by
+    the RIKV store as two calls, against the one call that writes the cache from the staged tiles."""
+    from oracle import regione_oracle as orc          # (row lists only; nothing is timed on the host)
+    wl = synth.WORKLOADS[3]
+    mask = synth.make_latents(wl, 0.25)["mask"][0]
+    rows = orc.region_rows(mask, wl.n_text, wl.n_ref, "edited_queries")["cache"]
+    qkv = synth.make_qkv_full(wl)
+    q, k, v = (to_dev(qkv[x]) for x in ("q", "k", "v"))
+    del qkv
+    n, H, D = wl.n_full, wl.heads, wl.head_dim
+    i32, bf = torch.int32, torch.bfloat16
+    keep = torch.zeros((1, n), dtype=i32, device="cuda"); keep[0, :len(rows)] = torch.from_numpy(rows).cuda()
+    n_keep = torch.tensor([len(rows)], dtype=i32, device="cuda")
+    n_rows = torch.tensor([n], dtype=i32, device="cuda"); zero = torch.zeros(1, dtype=i32, device="cuda")
+    kc = torch.empty((1, n, H, D), dtype=bf, device="cuda"); vc = torch.empty_like(kc)
+    out = torch.empty_like(q)
+    ws = torch.empty(max(binding.full_attention_store_workspace(1, n, H, D), 256), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=i32, device="cuda")
+
+    def two_calls():
+        binding.region_attention(q, k, v, None, None, n_rows, n_rows, zero, out, workspace=ws, dev_status=st)
+        binding.rikv_store(k, v, keep, n_keep, kc, vc, dev_status=st)
+
+    def one_call():
+        binding.full_attention_store(q, k, v, n_rows, keep, n_keep, kc, vc, out, workspace=ws, dev_status=st)
+
+    res = {}
+    for name, fn in (("attention_then_rikv_store_us", two_calls), ("full_attention_store_us", one_call)):
+        for _ in range(2):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        res[name] = round(float(np.median(ts)), 1)
+    assert int(st[0]) == 0
+    fl = 4.0 * H * D * n * n
+    res.update(workload="config 3 shape, forced full step with cache refresh", rows=n, kept_rows=len(rows),
+               full_attention_store_tflops=round(fl / res["full_attention_store_us"] / 1e6, 1),
+               frac_of_measured_burst=round(fl / res["full_attention_store_us"] / 1e6 / peaks["bf16_tflops"], 3))
+    return res
 
 
 def loop_row(torch, binding, synth, to_dev):

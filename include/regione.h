@@ -255,6 +255,36 @@ int regione_region_attention_scatter(const regione_bf16* q,
                                      int32_t* dev_status, void* stream);
 
 /*
+ * Full attention step that refreshes the Region-Instruction KV cache in passing (Sec. 4,
+ * "Stabilization Stage": the last full step saves K and V of every attention layer; end of the
+ * "Adaptive Velocity Decay Cache" paragraph: forced full-image steps update the cache; Algorithm 1,
+ * the store flag f[0] of a full DiT call).  One call does what
+ *     regione_region_attention(q, k, v, NULL, NULL, n_rows, n_rows, 0, ...)     (plain joint attention)
+ *     regione_rikv_store(k, v, keep_rows, n_keep, ...)
+ * do one after the other, bit for bit the same cache and the same output, but K and V are read from
+ * device memory once: the attention kernel stages every K / V tile of a head in shared memory anyway,
+ * and the thread block that walks the first query rows of a (request, head) writes the retained
+ * rows of each tile from there to their slots in the cache.
+ *
+ * q, k, v, out : dev bf16 [B, N_cap, H, D];  n_rows dev int32 [B] live rows (queries = keys)
+ * keep_rows    : dev int32 [B, Nc_cap], strictly ascending per request (as regione_region_rows
+ *                and regione_partition_rows write them); n_keep dev int32 [B]
+ * k_cache, v_cache : dev bf16 [B, Nc_cap, H, D]; rows past n_keep[b] are left untouched
+ * An entry of keep_rows outside [0, n_rows[b]) or out of order is skipped and REGIONE_DEV_BOUNDS
+ * recorded.  A request with n_rows[b] = 0 stores nothing.  Workspace: at least
+ * regione_full_attention_store_workspace(...) bytes, 256-byte aligned (it equals the query of
+ * regione_region_attention_workspace(B, N_cap, N_cap, 0, H, D)).  D must be 64 or 128.
+ */
+size_t regione_full_attention_store_workspace(int B, int N_cap, int H, int D);
+int regione_full_attention_store(const regione_bf16* q, const regione_bf16* k, const regione_bf16* v,
+                                 const int32_t* n_rows, int B, int N_cap, int H, int D,
+                                 float softmax_scale,
+                                 const int32_t* keep_rows, const int32_t* n_keep, int Nc_cap,
+                                 regione_bf16* k_cache, regione_bf16* v_cache, regione_bf16* out,
+                                 void* workspace, size_t workspace_bytes,
+                                 int32_t* dev_status, void* stream);
+
+/*
  * Region attention that brings its own scratch memory.  (The paper has no
  * counterpart: this entry point exists only for the way the library is deployed.)
  *

@@ -39,6 +39,9 @@ SIGNATURES = {
     "regione_region_attention_workspace": (c_size_t, [c_int] * 6),
     "regione_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, c_size_t, _P, _P]),
     "regione_region_attention_scatter": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, c_int, _P, _P, c_size_t, _P, _P]),
+    "regione_full_attention_store_workspace": (c_size_t, [c_int] * 4),
+    "regione_full_attention_store": (c_int, [_P] * 4 + [c_int] * 4 + [c_float, _P, _P, c_int, _P, _P, _P, _P,
+                                             c_size_t, _P, _P]),
     "regione_region_attention_static": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, _P]),
     "regione_avd_step": (c_int, [POINTER(c_double), c_double, c_double, c_double, POINTER(c_int)]),
     "regione_gamma_fit": (c_int, [_P, c_int, c_int, c_int64, _P, _P, _P, _P]),
@@ -275,6 +278,25 @@ def region_attention_scatter(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh
         _ptr(out_full, bf, "out_full"), out_full.shape[1], _ptr(out_rows, i32, "out_rows"),
         _ptr(workspace, None, "workspace"), ws_bytes, _ptr(dev_status, i32), _stream(stream)),
         "regione_region_attention_scatter")
+
+
+def full_attention_store_workspace(B, N_cap, H, D) -> int:
+    return int(load().regione_full_attention_store_workspace(B, N_cap, H, D))
+
+
+def full_attention_store(q, k, v, n_rows, keep_rows, n_keep, k_cache, v_cache, out, softmax_scale=0.0,
+                         workspace=None, dev_status=None, stream=None):
+    """Plain joint attention over q / k / v that also writes rows ``keep_rows`` of k and v to the cache."""
+    torch = _torch()
+    bf, i32 = torch.bfloat16, torch.int32
+    B, N_cap, H, D = q.shape
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().regione_full_attention_store(
+        _ptr(q, bf, "q"), _ptr(k, bf, "k"), _ptr(v, bf, "v"), _ptr(n_rows, i32, "n_rows"), B, N_cap, H, D,
+        float(softmax_scale), _ptr(keep_rows, i32, "keep_rows"), _ptr(n_keep, i32, "n_keep"),
+        keep_rows.shape[1], _ptr(k_cache, bf, "k_cache"), _ptr(v_cache, bf, "v_cache"), _ptr(out, bf, "out"),
+        _ptr(workspace, None, "workspace"), ws_bytes, _ptr(dev_status, i32), _stream(stream)),
+        "regione_full_attention_store")
 
 
 def region_attention_static(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, out,

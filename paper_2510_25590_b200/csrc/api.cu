@@ -13,7 +13,7 @@ size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, 
 int launch_region_attention_tc(const uint16_t*, const uint16_t*, const uint16_t*, const uint16_t*,
                                const uint16_t*, const int32_t*, const int32_t*, const int32_t*, int,
                                int, int, int, int, int, float, uint16_t*, const int32_t*, int, void*,
-                               size_t, int32_t*, cudaStream_t);
+                               size_t, int32_t*, cudaStream_t, const CacheStore*);
 }  // namespace regione
 
 using namespace regione;
@@ -94,7 +94,7 @@ static int region_attention_impl(const regione_bf16* q, const regione_bf16* k_fr
     }
     return launch_region_attention_tc(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
                                       B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, out_rows, out_cap,
-                                      workspace, workspace_bytes, dev_status, (cudaStream_t)stream);
+                                      workspace, workspace_bytes, dev_status, (cudaStream_t)stream, nullptr);
 }
 
 extern "C" int regione_region_attention(const regione_bf16* q, const regione_bf16* k_fresh,
@@ -119,6 +119,38 @@ extern "C" int regione_region_attention_scatter(
     return region_attention_impl(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache, B,
                                  Nq_cap, Nf_cap, Nc_cap, H, D, softmax_scale, out_full, out_rows,
                                  out_rows_cap, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" size_t regione_full_attention_store_workspace(int B, int N_cap, int H, int D) {
+    return regione_region_attention_workspace(B, N_cap, N_cap, 0, H, D);
+}
+
+extern "C" int regione_full_attention_store(
+    const regione_bf16* q, const regione_bf16* k, const regione_bf16* v, const int32_t* n_rows, int B,
+    int N_cap, int H, int D, float softmax_scale, const int32_t* keep_rows, const int32_t* n_keep,
+    int Nc_cap, regione_bf16* k_cache, regione_bf16* v_cache, regione_bf16* out, void* workspace,
+    size_t workspace_bytes, int32_t* dev_status, void* stream) {
+    bool nothing = false;
+    const int rc = check_attention_args(q, k, v, nullptr, nullptr, n_rows, n_rows, n_rows, B, N_cap, N_cap,
+                                        0, H, D, out, &nothing);
+    if (rc != REGIONE_OK) return rc;
+    if (!keep_rows || !n_keep || Nc_cap < 0) return REGIONE_INVALID_ARG;
+    if (Nc_cap > 0 && (!k_cache || !v_cache)) return REGIONE_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache)) return REGIONE_INVALID_ARG;
+    if (nothing || N_cap == 0) return REGIONE_OK;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    const size_t need = region_attention_tc_workspace(B, N_cap, N_cap, 0, H, D);
+    if (need > 0) {
+        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return REGIONE_INVALID_ARG;
+        if (workspace_bytes < need) return REGIONE_WORKSPACE_TOO_SMALL;
+    }
+    CacheStore store;
+    store.keep_rows = keep_rows; store.n_keep = n_keep; store.cap = Nc_cap;
+    store.k_cache = k_cache; store.v_cache = v_cache;
+    // no cached segment: n_cache = nullptr stands for "zero rows" in every request
+    return launch_region_attention_tc(q, k, v, nullptr, nullptr, n_rows, n_rows, nullptr, B, N_cap, N_cap, 0,
+                                      H, D, scale, out, nullptr, 0, workspace, workspace_bytes, dev_status,
+                                      (cudaStream_t)stream, Nc_cap > 0 ? &store : nullptr);
 }
 
 // The CUDA-core kernel, reachable only through this symbol: an independent arithmetic path on the

@@ -11,8 +11,10 @@
 //              are two tensor maps walked one after the other
 //   warps 9,10 tcgen05.mma issuers, one per query tile (the whole warp walks the
 //              loop, one elected lane issues); warp 9 owns the tensor-memory allocation
-//   warp  11   idle (fills the third warpgroup so that registers can be moved from
-//              it to the softmax warpgroups with setmaxnreg)
+//   warp  11   fills the third warpgroup so that registers can be moved from it to the
+//              softmax warpgroups with setmaxnreg; idle, except in the full step that
+//              refreshes the Region-Instruction KV cache: there it copies the retained rows of
+//              every staged K / V tile from shared memory to their places in the cache
 //
 // Tensor memory (512 columns): S0 | S1 | O0 | O1.  S_t = Q_t K_j^T (fp32, 128
 // columns) is read back by the softmax warps of tile t, the probabilities are
@@ -124,6 +126,13 @@ struct AttnParams {
     float2* part_ml;     // [B, H, P_cap, max_slots, 256]    (running max in the exp2 domain, sum)
     CutItem* cut;        // [grid] the item that the start of each share cuts, for the merge kernel
     long long timeout_cycles;   // bound of every barrier wait, in SM clock cycles
+    // Cache refresh fused into a full step (all nullptr / 0 otherwise): the rows keep_rows[b, 0..n_keep[b])
+    // (ascending) of the fresh K and V are also written to k_store / v_store [B, store_cap, H, D].
+    const int32_t* keep_rows;
+    const int32_t* n_keep;
+    int store_cap;
+    uint16_t* k_store;
+    uint16_t* v_store;
 };
 
 
@@ -145,9 +154,11 @@ struct ReqShape {
     long long ticks_full, ticks_last, head_ticks, ticks;   // per full-pair item, last item, head, request
 };
 
+// NO_CACHE: the launch has no cached segment at all (p.n_cache is not read).
+template <bool NO_CACHE>
 __device__ __forceinline__ ReqShape req_shape(const AttnParams& p, int b, bool* bad = nullptr) {
     ReqShape r;
-    int nq = p.n_q[b], nf = p.n_fresh[b], nc = p.n_cache[b];
+    int nq = p.n_q[b], nf = p.n_fresh[b], nc = NO_CACHE ? 0 : p.n_cache[b];
     if (nq < 0 || nq > p.Nq_cap || nf < 0 || nf > p.Nf_cap || nc < 0 || nc > p.Nc_cap) {
         if (bad) *bad = true;
         nq = max(0, min(nq, p.Nq_cap));
@@ -179,11 +190,12 @@ struct Plan {
     long long total, chunk;
 };
 
+template <bool NO_CACHE>
 __device__ __forceinline__ Plan plan_shares(const AttnParams& p, int grid, bool* bad = nullptr) {
     Plan pl;
     long long items = 0, ticks = 0, span = 0;      // span: first tick of an item's last step, at most
     for (int b = 0; b < p.B; ++b) {
-        const ReqShape r = req_shape(p, b, bad);
+        const ReqShape r = req_shape<NO_CACHE>(p, b, bad);
         items += r.items;
         ticks += r.ticks;
         if (r.np > 0) span = max(span, (long long)(r.np > 1 ? kTickPair : r.w_last) * (r.steps - 1));
@@ -230,15 +242,16 @@ __device__ __forceinline__ void item_slots(const Plan& pl, long long first_tick,
 }
 
 // Whole-item plan: the item with index `idx`.
+template <bool NO_CACHE>
 __device__ __forceinline__ Segment segment_whole(const AttnParams& p, long long idx) {
     Segment sg;
     long long base = 0;
     int b = 0;
-    ReqShape r = req_shape(p, 0);
+    ReqShape r = req_shape<NO_CACHE>(p, 0);
     while (idx >= base + r.items && b + 1 < p.B) {
         base += r.items;
         ++b;
-        r = req_shape(p, b);
+        r = req_shape<NO_CACHE>(p, b);
     }
     const long long item = idx - base;
     sg.b = b; sg.r = r;
@@ -252,16 +265,17 @@ __device__ __forceinline__ Segment segment_whole(const AttnParams& p, long long 
 }
 
 // Tick plan: the item that contains tick `pos`, and the steps of it that share `c` owns.
+template <bool NO_CACHE>
 __device__ __forceinline__ Segment segment_ticks(const AttnParams& p, const Plan& pl, long long pos,
                                                  int c) {
     Segment sg;
     long long base = 0;
     int b = 0;
-    ReqShape r = req_shape(p, 0);
+    ReqShape r = req_shape<NO_CACHE>(p, 0);
     while (pos >= base + r.ticks && b + 1 < p.B) {
         base += r.ticks;
         ++b;
-        r = req_shape(p, b);
+        r = req_shape<NO_CACHE>(p, b);
     }
     sg.b = b; sg.r = r;
     if (r.np == 0) {                                  // nothing left behind the last live request
@@ -363,7 +377,9 @@ __device__ __forceinline__ float chunk_probabilities(uint32_t tP, const uint32_t
 // (SOFTMAX_WG, many registers) or the producer / issuer warpgroup (few).  The two instantiations
 // are called from the two sides of the setmaxnreg split so that each is compiled for its own
 // register budget; both execute the same sequence of CTA-wide barriers.
-template <int D, bool SOFTMAX_WG>
+// STORE: the instantiation for the full step that also refreshes the cache (warp 11 writes the
+// retained K / V rows); the plain instantiation contains none of that code.
+template <int D, bool SOFTMAX_WG, bool STORE>
 __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtensorMap* tm_kf_,
                                           const CUtensorMap* tm_vf_, const CUtensorMap* tm_kc_,
                                           const CUtensorMap* tm_vc_, const AttnParams& p,
@@ -382,7 +398,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     bool first_segment = true;
     while (pos < hi) {
     // ---- the segment: key tiles [j_first, j_first + n_tiles) of item (b, h, query pair) ----
-    const Segment it = pl.whole_items ? segment_whole(p, pos) : segment_ticks(p, pl, pos, (int)blockIdx.x);
+    const Segment it = pl.whole_items ? segment_whole<STORE>(p, pos)
+                                      : segment_ticks<STORE>(p, pl, pos, (int)blockIdx.x);
     if (first_segment && SOFTMAX_WG && threadIdx.x == 0) {
         // tell the merge kernel which item the start of this share cuts
         CutItem ci;
@@ -414,6 +431,9 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     // a lone tile's ring starts at the idle second query tile and runs over the extra stage: two
     // stages more, because its two halves consume K/V tiles at twice the rate per chain
     const int n_stages = split ? kStages + 2 : kStages;
+    // cache refresh: the first query pair of every (request, head) also writes the retained rows of
+    // the key tiles it walks, so every (request, head, key tile) is written exactly once
+    const bool store_item = STORE && p.keep_rows != nullptr && it.qp == 0 && n_tiles > 0;
     const uint32_t ring = split ? sQ + kTileBytes : sKV;
     uint8_t* const ring_gen = smem_gen + (split ? 1 : 2) * kTileBytes;
 
@@ -421,7 +441,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     if (threadIdx.x < kNumBarriers) {
         const int i = threadIdx.x;
         int count = 1;                                               // q_full, kv_full, s_full, o_final
-        if (i >= kBarKvEmpty && i < kBarSFull) count = split ? 1 : ntq;             // commits per stage
+        if (i >= kBarKvEmpty && i < kBarSFull) count = (split ? 1 : ntq) + (store_item ? 1 : 0);   // commits per stage (+ the cache writer)
         else if ((i >= kBarPFull && i < kBarOFinal) || i >= kBarTurn) count = kBM / 32;   // one arrival per warp
         ptx::mbar_init(ptx::smem_addr(&ctrl->q_full + i), count);
         ptx::fence_barrier_init();
@@ -478,6 +498,83 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 for (int hf = 0; hf < Cfg::kHalves; ++hf)
                     ptx::tma_load_4d(ring + stage * kTileBytes + hf * kHalfBytes, map, bar, hf * 64, h,
                                      row0, b);
+            }
+        }
+    } else if (STORE && warp == 11) {
+        // ================= cache writer (full step that refreshes the RIKV cache) =================
+        if (store_item) {
+            constexpr int kCpr = D / 8;                 // 16-byte chunks per row of one head
+            constexpr int kRowsPer = 32 / kCpr;         // rows a warp instruction moves
+            const int32_t* keep = p.keep_rows + (size_t)b * p.store_cap;
+            int nk = p.n_keep[b];
+            if (nk < 0 || nk > p.store_cap) {
+                record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+                nk = max(0, min(nk, p.store_cap));
+            }
+            // first retained row at or behind this segment's first key row: 32-ary search, one
+            // coalesced probe per level
+            const int row_first = j_first * kBN;        // (a full step has no cached segment)
+            int lo = 0, len = nk;
+            while (len > 0) {
+                const int step = (len + 31) / 32;
+                const int at = lo + min(lane * step, len - 1);
+                const bool below = (lane * step < len) && keep[at] < row_first;
+                const int nb = __popc(__ballot_sync(0xffffffffu, below));   // probes below the target
+                // the answer lies behind probe nb - 1 and at or before probe nb
+                const int new_lo = nb == 0 ? lo : lo + (nb - 1) * step + 1;
+                const int new_hi = nb == 0 ? lo : min(lo + nb * step, lo + len);
+                len = (step == 1) ? 0 : new_hi - new_lo;
+                lo = (step == 1) ? lo + nb : new_lo;
+            }
+            bool ok = true;
+            for (int jl = 0; jl < n_tiles && ok; ++jl) {
+                bool cached; int row0, valid;
+                tile_seg(jl, cached, row0, valid);
+                // retained rows of this tile: at most kBN consecutive entries of the ascending list
+                int r[kBN / 32];
+                int cnt = 0;                            // length of the run of entries inside this tile
+                bool run_open = true;
+#pragma unroll
+                for (int k = 0; k < kBN / 32; ++k) {
+                    const int i = lo + k * 32 + lane;
+                    r[k] = i < nk ? keep[i] - row0 : kBN;
+                    if (r[k] < 0) {                     // the list is not ascending
+                        record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+                        r[k] = kBN;
+                    }
+                    const uint32_t inside = __ballot_sync(0xffffffffu, r[k] < valid);
+                    if (run_open) cnt += inside == 0xffffffffu ? 32 : __ffs(~inside) - 1;
+                    run_open = run_open && inside == 0xffffffffu;
+                }
+                for (int is_v = 0; is_v < 2 && ok; ++is_v) {
+                    const int i_ring = 2 * jl + is_v, stage = i_ring % n_stages;
+                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[stage]), (i_ring / n_stages) & 1, abort_flag,
+                                  p.dev_status, p.timeout_cycles);
+                    if (!ok) break;
+                    const uint8_t* tile = ring_gen + stage * kTileBytes;
+                    uint16_t* dst_base = (is_v ? p.v_store : p.k_store) +
+                                         (((size_t)b * p.store_cap + lo) * p.H + h) * D;
+                    const int q = lane % kCpr;          // this lane's 16-byte chunk of the row
+#pragma unroll
+                    for (int k = 0; k < kBN / 32; ++k) {
+                        if (k * 32 >= cnt) break;                       // (uniform)
+#pragma unroll 2
+                        for (int e1 = 0; e1 < 32; e1 += kRowsPer) {
+                            const int el = e1 + lane / kCpr;            // entry of the tile's run: k * 32 + el
+                            const int rr = __shfl_sync(0xffffffffu, r[k], el);
+                            if (k * 32 + el < cnt) {
+                                const uint4 x = *reinterpret_cast<const uint4*>(
+                                    tile + (q >> 3) * kHalfBytes + rr * 128 + (((q & 7) ^ (rr & 7)) << 4));
+                                *reinterpret_cast<uint4*>(dst_base + (size_t)(k * 32 + el) * p.H * D + q * 8) = x;
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->kv_empty[stage]));
+                }
+                lo += cnt;
+                // entries left over behind the item's last key tile name rows that do not exist
+                if (j_first + jl == it.r.nt - 1 && lo < nk) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
             }
         }
     } else if (warp == 9 || warp == 10) {
@@ -816,7 +913,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     }   // segments
 }
 
-template <int D>
+template <int D, bool STORE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                            const __grid_constant__ CUtensorMap tm_kf,
@@ -838,7 +935,7 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     grid_dependency_wait();                             // (everything below reads the launch's inputs)
     // this CTA's share [pos, hi) of the item sequence or of the cost axis
     bool bad = false;
-    const Plan pl = plan_shares(p, gridDim.x, &bad);
+    const Plan pl = plan_shares<STORE>(p, gridDim.x, &bad);
     if (bad && blockIdx.x == 0 && threadIdx.x == 0) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
     // (whole items are dealt round-robin, so that the CTAs running at any one time work on
     // neighbouring items, which share K/V tiles in L2; a share of steps is one contiguous range)
@@ -857,11 +954,11 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
     if (warp >= 8) {
         ptx::reg_dealloc<56>();                         // producer / issuer warpgroup gives registers up
-        run_share<D, false>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
+        run_share<D, false, STORE>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
                             sKV, warp, lane);
     } else {
         ptx::reg_alloc<224>();                          // a row of 128 logits stays in registers
-        run_share<D, true>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
+        run_share<D, true, STORE>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
                            sKV, warp, lane);
     }
 
@@ -1069,24 +1166,32 @@ size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, 
            ((rows * sizeof(float2) + 255) & ~(size_t)255) + (size_t)lp.grid * sizeof(CutItem);
 }
 
-template <int D>
-static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, cudaStream_t st) {
+template <int D, bool STORE>
+static int launch_main(const CUtensorMap* maps, const AttnParams& prm, int grid, cudaStream_t st) {
     using Cfg = AttnCfg<D>;
     // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
     static int configured[kMaxDevices] = {};
     const int dev = current_device();
     if (dev < 0) return REGIONE_CUDA_ERROR;
     if (!__atomic_load_n(&configured[dev], __ATOMIC_ACQUIRE)) {
-        if (cudaFuncSetAttribute(region_attention_tc_kernel<D>,
+        if (cudaFuncSetAttribute(region_attention_tc_kernel<D, STORE>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg::kSmemBytes) != cudaSuccess)
             return REGIONE_CUDA_ERROR;
         __atomic_store_n(&configured[dev], 1, __ATOMIC_RELEASE);
     }
-    if (launch_overlapped(region_attention_tc_kernel<D>, dim3(grid), dim3(kAttnThreads),
+    if (launch_overlapped(region_attention_tc_kernel<D, STORE>, dim3(grid), dim3(kAttnThreads),
                           Cfg::kSmemBytes, st, maps[0], maps[1], maps[2], maps[3], maps[4],
                           prm) != cudaSuccess)
         return REGIONE_CUDA_ERROR;
+    return REGIONE_OK;
+}
+
+template <int D>
+static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, cudaStream_t st) {
+    const int rc = prm.keep_rows != nullptr ? launch_main<D, true>(maps, prm, grid, st)
+                                            : launch_main<D, false>(maps, prm, grid, st);
+    if (rc != REGIONE_OK) return rc;
     // the merge kernel may become resident while the attention kernel drains (it waits for that
     // kernel's completion before it reads a slot)
     if (grid < 2) return launch_status(cudaGetLastError());     // a single share cuts nothing
@@ -1109,7 +1214,8 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
                                const int32_t* n_fresh, const int32_t* n_cache, int B, int Nq_cap,
                                int Nf_cap, int Nc_cap, int H, int D, float scale, uint16_t* out,
                                const int32_t* out_rows, int out_cap, void* workspace,
-                               size_t workspace_bytes, int32_t* dev_status, cudaStream_t st) {
+                               size_t workspace_bytes, int32_t* dev_status, cudaStream_t st,
+                               const CacheStore* store) {
     (void)workspace_bytes;
     CUtensorMap maps[5];
     // an absent segment still needs a valid (never dereferenced) base address
@@ -1131,6 +1237,11 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
     prm.out_rows = out_rows;
     prm.out_cap = out_rows != nullptr ? out_cap : Nq_cap;
     prm.timeout_cycles = kTimeoutCycles;
+    prm.keep_rows = store != nullptr ? store->keep_rows : nullptr;
+    prm.n_keep = store != nullptr ? store->n_keep : nullptr;
+    prm.store_cap = store != nullptr ? store->cap : 0;
+    prm.k_store = store != nullptr ? store->k_cache : nullptr;
+    prm.v_store = store != nullptr ? store->v_cache : nullptr;
     const size_t rows = slot_rows(lp, B, H);
     prm.part_o = reinterpret_cast<float*>(workspace);
     uint8_t* const ws = reinterpret_cast<uint8_t*>(workspace);
@@ -1200,5 +1311,5 @@ extern "C" int regione_region_attention_static(
     // by the attention kernel of the same call, so the previous call's contents are harmless.
     return launch_region_attention_tc(q, k_fresh, v_fresh, k_cache, v_cache, n_q, n_fresh, n_cache,
                                       B, Nq_cap, Nf_cap, Nc_cap, H, D, scale, out, nullptr, 0, scratch,
-                                      kStaticScratchBytes, dev_status, (cudaStream_t)stream);
+                                      kStaticScratchBytes, dev_status, (cudaStream_t)stream, nullptr);
 }

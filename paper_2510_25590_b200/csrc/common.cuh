@@ -81,6 +81,15 @@ struct PerRequestF {
     float v[kReqChunk];
 };
 
+// The cache refresh a full attention step can carry along (regione_full_attention_store).
+struct CacheStore {
+    const int32_t* keep_rows;   // dev [B, cap], ascending per request
+    const int32_t* n_keep;      // dev [B]
+    int cap;
+    uint16_t* k_cache;          // dev [B, cap, H, D]
+    uint16_t* v_cache;
+};
+
 // Host-side argument checks shared by every region-attention entry point (defined in api.cu).
 // Returns REGIONE_OK when the call may proceed; *nothing_to_do is set for B == 0 or Nq_cap == 0.
 int check_attention_args(const void* q, const void* k_fresh, const void* v_fresh, const void* k_cache,
