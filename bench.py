@@ -370,17 +370,23 @@ def full_step_row(torch, binding, synth, flush_l2, to_dev, peaks, iters=10):
     """The forced full step on the Qwen-Image-Edit-shaped layer (8448 joint rows, 24 heads x 128, the
     cache keeps text + unedited + reference rows of the 25 % mask): plain joint attention followed by
     the RIKV store as two calls, against the one call that writes the cache from the staged tiles."""
-    from oracle import regione_oracle as orc          # (row lists only; nothing is timed on the host)
     wl = synth.WORKLOADS[3]
-    mask = synth.make_latents(wl, 0.25)["mask"][0]
-    rows = orc.region_rows(mask, wl.n_text, wl.n_ref, "edited_queries")["cache"]
+    lat = synth.make_latents(wl, 0.25)
     qkv = synth.make_qkv_full(wl)
     q, k, v = (to_dev(qkv[x]) for x in ("q", "k", "v"))
     del qkv
-    n, H, D = wl.n_full, wl.heads, wl.head_dim
+    n, H, D, N = wl.n_full, wl.heads, wl.head_dim, wl.n_img
     i32, bf = torch.int32, torch.bfloat16
-    keep = torch.zeros((1, n), dtype=i32, device="cuda"); keep[0, :len(rows)] = torch.from_numpy(rows).cuda()
-    n_keep = torch.tensor([len(rows)], dtype=i32, device="cuda")
+    # the rows to retain come from the library's own partition and row lists
+    mask = torch.empty((1, N), dtype=torch.uint8, device="cuda")
+    e_idx, k_idx, slot = (torch.empty((1, N), dtype=i32, device="cuda") for _ in range(3))
+    n_edit, n_query, n_keep = (torch.zeros(1, dtype=i32, device="cuda") for _ in range(3))
+    query_rows = torch.zeros((1, n), dtype=i32, device="cuda")
+    keep = torch.zeros((1, n), dtype=i32, device="cuda")
+    binding.partition_rows(to_dev(lat["x_t"]), to_dev(lat["v"]), to_dev(lat["ref"]), lat["t"],
+                           binding.METRIC_COSINE, wl.threshold, mask, e_idx, k_idx, slot, n_edit,
+                           wl.n_text, wl.n_ref, binding.ROWS_EDITED_QUERIES, query_rows, n_query, keep, n_keep)
+    kept = int(n_keep[0])
     n_rows = torch.tensor([n], dtype=i32, device="cuda"); zero = torch.zeros(1, dtype=i32, device="cuda")
     kc = torch.empty((1, n, H, D), dtype=bf, device="cuda"); vc = torch.empty_like(kc)
     out = torch.empty_like(q)
@@ -408,7 +414,7 @@ def full_step_row(torch, binding, synth, flush_l2, to_dev, peaks, iters=10):
         res[name] = round(float(np.median(ts)), 1)
     assert int(st[0]) == 0
     fl = 4.0 * H * D * n * n
-    res.update(workload="config 3 shape, forced full step with cache refresh", rows=n, kept_rows=len(rows),
+    res.update(workload="config 3 shape, forced full step with cache refresh", rows=n, kept_rows=kept,
                full_attention_store_tflops=round(fl / res["full_attention_store_us"] / 1e6, 1),
                frac_of_measured_burst=round(fl / res["full_attention_store_us"] / 1e6 / peaks["bf16_tflops"], 3))
     return res

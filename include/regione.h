@@ -33,7 +33,11 @@
  *    may sit at its own sampler step: the sampler scalars (t, dt, scale,
  *    dt_unedited) are host arrays of B floats, read during the call (the
  *    values travel to the kernels as launch parameters, 128 requests per
- *    launch; the arrays may be reused as soon as the call returns).
+ *    launch; the arrays may be reused as soon as the call returns).  A request
+ *    whose scalar is NaN (t for the partition, dt or scale for the velocity
+ *    decay, dt_unedited for the merge) sits that call out: nothing of it is
+ *    read or written.  This is how a batch whose requests are at different
+ *    kinds of step shares one launch.
  *  - There is no CPU fallback: without a CUDA device every compute entry point
  *    returns REGIONE_CUDA_ERROR.
  */

@@ -29,6 +29,7 @@ velocity_decay_kernel(const uint4* __restrict__ v_in, const PerRequestF neg_dt_s
     grid_launch_dependents();
     const int b = b0 + blockIdx.y;                       // requests b0 .. b0 + gridDim.y of the batch
     const float neg_dt_scale = neg_dt_scale_v.v[blockIdx.y];
+    if (neg_dt_scale != neg_dt_scale) return;            // NaN: this request sits the call out
     int ne = n_edit[b];
     if (ne < 0 || ne > Ne_cap) {
         if (threadIdx.x == 0 && blockIdx.x == 0) record_status(dev_status, REGIONE_DEV_BOUNDS);
@@ -58,6 +59,7 @@ merge_kernel(const uint4* x_full, const uint4* __restrict__ v_last,
     grid_launch_dependents();
     const int b = b0 + blockIdx.y;
     const float neg_dt = neg_dt_v.v[blockIdx.y];
+    if (neg_dt != neg_dt) return;                        // NaN: this request sits the call out
     const unsigned total = (unsigned)N * (unsigned)cpr;
     const unsigned base = blockIdx.x * (unsigned)(kLatThreads * kMergeUnroll) + threadIdx.x;
     const size_t req = (size_t)b * N * cpr;

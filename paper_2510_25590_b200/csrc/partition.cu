@@ -145,6 +145,7 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
     const int csize = cluster.num_blocks();
     const int b = b0 + blockIdx.y;               // this launch covers requests b0 .. b0 + gridDim.y
     const float t = tv.v[blockIdx.y];            // the request's own sampler time
+    if (t != t) return;                          // NaN: this request sits the call out (whole cluster)
     const int start = rank * share;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int TPI = 32 / L;                 // tokens per sub-iteration

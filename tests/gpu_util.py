@@ -33,6 +33,8 @@ def errors(got, want):
     got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
     ok = np.isfinite(want)
     d = got[ok] - want[ok]
+    if d.size == 0:
+        return 0.0, 0.0
     rms = np.sqrt(np.mean(want[ok] ** 2))
     return float(np.max(np.abs(d))) if d.size else 0.0, float(np.sqrt(np.mean(d * d)) / rms) if d.size and rms > 0 else 0.0
 

@@ -105,3 +105,35 @@ def test_step_replayed_from_a_cuda_graph_matches_the_eager_step():
     for n in names:
         a, b = eager[n], getattr(step, n)
         assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), n
+
+
+def test_guidance_pair_two_batch_entries_sharing_one_mask():
+    """Classifier-free guidance evaluates the model twice per step (the paper's editors run with guidance
+    scales 6, 2.5 and 4): the conditional and the unconditional branch are two batch entries with the same
+    latent, hence the same edit mask and index lists, but their own Q / K / V.  One launch of every stage
+    serves both; each entry must match the oracle on its own inputs."""
+    import torch
+    base = synth.scaled_workload(synth.WORKLOADS[2], grid=(24, 24), n_text=40, heads=3)
+    wl = synth.scaled_workload(base, batch=2)
+    one = synth.make_latents(base)
+    lat = {k: (np.concatenate([one[k], one[k]]) if isinstance(one[k], np.ndarray) else one[k]) for k in one}
+    qkv = synth.make_qkv_full(wl)                       # two different Q / K / V sets
+    assert not np.array_equal(qkv["q"][0], qkv["q"][1])
+    t, scale, dt, dt_u = lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0
+    d = {k: dev_bf16(lat[k]) for k in ("x_t", "v", "ref")}
+    dq, dk, dv = (dev_bf16(qkv[k]) for k in ("q", "k", "v"))
+    cap = plan_capacity(d["x_t"], d["v"], d["ref"], t, binding.METRIC_COSINE, wl.threshold)
+    step = RegionStep(StepShapes(2, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads, wl.head_dim, cap,
+                                 binding.METRIC_COSINE, wl.threshold, binding.ROWS_EDITED_QUERIES))
+    step.run(d["x_t"], d["v"], d["ref"], dq, dk, dv, t, scale, dt, dt_u)
+    torch.cuda.synchronize()
+    assert int(step.dev_status[0]) == 0
+    assert torch.equal(step.mask[0], step.mask[1]) and torch.equal(step.query_rows[0], step.query_rows[1])
+    assert int(step.n_q[0]) == int(step.n_q[1]) > 0
+    want = step_oracle.region_step(wl, lat, qkv, t, np.float32(scale), np.float32(dt), np.float32(dt_u))
+    for b in range(2):
+        nq = int(want["n_q"][b])
+        rows = step.query_rows[b, :nq].long()
+        assert_close(host_f64(step.o_full[b][rows]), want["o_e"][b, :nq], f"guidance branch {b}")
+    assert not torch.equal(step.o_full[0], step.o_full[1])
+    assert_close(host_f64(step.x_out), want["x_out"], "merged latents")
