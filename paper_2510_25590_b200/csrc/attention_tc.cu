@@ -126,8 +126,12 @@ struct AttnParams {
     float2* part_ml;     // [B, H, P_cap, max_slots, 256]    (running max in the exp2 domain, sum)
     CutItem* cut;        // [grid] the item that the start of each share cuts, for the merge kernel
     long long timeout_cycles;   // bound of every barrier wait, in SM clock cycles
-    // Cache refresh fused into a full step (all nullptr / 0 otherwise): the rows keep_rows[b, 0..n_keep[b])
-    // (ascending) of the fresh K and V are also written to k_store / v_store [B, store_cap, H, D].
+};
+
+// Cache refresh fused into a full step: the rows keep_rows[b, 0..n_keep[b]) (ascending) of the fresh
+// K and V are also written to k_store / v_store [B, store_cap, H, D].  A parameter of its own, of
+// the kernel that refreshes the cache only: the plain attention kernel's parameters do not grow.
+struct StoreParams {
     const int32_t* keep_rows;
     const int32_t* n_keep;
     int store_cap;
@@ -383,6 +387,7 @@ template <int D, bool SOFTMAX_WG, bool STORE>
 __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtensorMap* tm_kf_,
                                           const CUtensorMap* tm_vf_, const CUtensorMap* tm_kc_,
                                           const CUtensorMap* tm_vc_, const AttnParams& p,
+                                          const StoreParams& sp,
                                           long long pos, const long long hi, const Plan pl,
                                           AttnCtrl* ctrl, uint8_t* smem_gen, const uint32_t sQ,
                                           const uint32_t sKV, const int warp, const int lane) {
@@ -433,7 +438,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     const int n_stages = split ? kStages + 2 : kStages;
     // cache refresh: the first query pair of every (request, head) also writes the retained rows of
     // the key tiles it walks, so every (request, head, key tile) is written exactly once
-    const bool store_item = STORE && p.keep_rows != nullptr && it.qp == 0 && n_tiles > 0;
+    const bool store_item = STORE && it.qp == 0 && n_tiles > 0;
     const uint32_t ring = split ? sQ + kTileBytes : sKV;
     uint8_t* const ring_gen = smem_gen + (split ? 1 : 2) * kTileBytes;
 
@@ -505,11 +510,11 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         if (store_item) {
             constexpr int kCpr = D / 8;                 // 16-byte chunks per row of one head
             constexpr int kRowsPer = 32 / kCpr;         // rows a warp instruction moves
-            const int32_t* keep = p.keep_rows + (size_t)b * p.store_cap;
-            int nk = p.n_keep[b];
-            if (nk < 0 || nk > p.store_cap) {
+            const int32_t* keep = sp.keep_rows + (size_t)b * sp.store_cap;
+            int nk = sp.n_keep[b];
+            if (nk < 0 || nk > sp.store_cap) {
                 record_status(p.dev_status, REGIONE_DEV_BOUNDS);
-                nk = max(0, min(nk, p.store_cap));
+                nk = max(0, min(nk, sp.store_cap));
             }
             // first retained row at or behind this segment's first key row: 32-ary search, one
             // coalesced probe per level
@@ -552,8 +557,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                                   p.dev_status, p.timeout_cycles);
                     if (!ok) break;
                     const uint8_t* tile = ring_gen + stage * kTileBytes;
-                    uint16_t* dst_base = (is_v ? p.v_store : p.k_store) +
-                                         (((size_t)b * p.store_cap + lo) * p.H + h) * D;
+                    uint16_t* dst_base = (is_v ? sp.v_store : sp.k_store) +
+                                         (((size_t)b * sp.store_cap + lo) * p.H + h) * D;
                     const int q = lane % kCpr;          // this lane's 16-byte chunk of the row
 #pragma unroll
                     for (int k = 0; k < kBN / 32; ++k) {
@@ -914,12 +919,10 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
 }
 
 template <int D, bool STORE>
-__global__ void __launch_bounds__(kAttnThreads, 1)
-region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
-                           const __grid_constant__ CUtensorMap tm_kf,
-                           const __grid_constant__ CUtensorMap tm_vf,
-                           const __grid_constant__ CUtensorMap tm_kc,
-                           const __grid_constant__ CUtensorMap tm_vc, const AttnParams p) {
+__device__ __forceinline__ void attention_kernel_body(const CUtensorMap& tm_q, const CUtensorMap& tm_kf,
+                                                      const CUtensorMap& tm_vf, const CUtensorMap& tm_kc,
+                                                      const CUtensorMap& tm_vc, const AttnParams& p,
+                                                      const StoreParams& sp) {
     using Cfg = AttnCfg<D>;
     constexpr int kTileBytes = Cfg::kTileBytes;
 
@@ -954,12 +957,12 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
     if (warp >= 8) {
         ptx::reg_dealloc<56>();                         // producer / issuer warpgroup gives registers up
-        run_share<D, false, STORE>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
-                            sKV, warp, lane);
+        run_share<D, false, STORE>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, sp, pos, hi, pl, ctrl, smem_gen,
+                                   sQ, sKV, warp, lane);
     } else {
         ptx::reg_alloc<224>();                          // a row of 128 logits stays in registers
-        run_share<D, true, STORE>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, pos, hi, pl, ctrl, smem_gen, sQ,
-                           sKV, warp, lane);
+        run_share<D, true, STORE>(&tm_q, &tm_kf, &tm_vf, &tm_kc, &tm_vc, p, sp, pos, hi, pl, ctrl, smem_gen,
+                                  sQ, sKV, warp, lane);
     }
 
     // ================= teardown =================
@@ -975,6 +978,28 @@ region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(ctrl->tmem_base, 512);
     }
+}
+
+// The attention kernel, and the one that also refreshes the cache (one parameter more).
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+region_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
+                           const __grid_constant__ CUtensorMap tm_kf,
+                           const __grid_constant__ CUtensorMap tm_vf,
+                           const __grid_constant__ CUtensorMap tm_kc,
+                           const __grid_constant__ CUtensorMap tm_vc, const AttnParams p) {
+    const StoreParams none = {};
+    attention_kernel_body<D, false>(tm_q, tm_kf, tm_vf, tm_kc, tm_vc, p, none);
+}
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+region_attention_store_kernel(const __grid_constant__ CUtensorMap tm_q,
+                              const __grid_constant__ CUtensorMap tm_kf,
+                              const __grid_constant__ CUtensorMap tm_vf,
+                              const __grid_constant__ CUtensorMap tm_kc,
+                              const __grid_constant__ CUtensorMap tm_vc, const AttnParams p,
+                              const StoreParams sp) {
+    attention_kernel_body<D, true>(tm_q, tm_kf, tm_vf, tm_kc, tm_vc, p, sp);
 }
 
 // Merges the workspace slots of the items that were spread over several shares:
@@ -1167,30 +1192,38 @@ size_t region_attention_tc_workspace(int B, int Nq_cap, int Nf_cap, int Nc_cap, 
 }
 
 template <int D, bool STORE>
-static int launch_main(const CUtensorMap* maps, const AttnParams& prm, int grid, cudaStream_t st) {
+static int launch_main(const CUtensorMap* maps, const AttnParams& prm, const StoreParams& sp, int grid,
+                       cudaStream_t st) {
     using Cfg = AttnCfg<D>;
     // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
     static int configured[kMaxDevices] = {};
     const int dev = current_device();
     if (dev < 0) return REGIONE_CUDA_ERROR;
     if (!__atomic_load_n(&configured[dev], __ATOMIC_ACQUIRE)) {
-        if (cudaFuncSetAttribute(region_attention_tc_kernel<D, STORE>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg::kSmemBytes) != cudaSuccess)
-            return REGIONE_CUDA_ERROR;
+        const cudaError_t e =
+            STORE ? cudaFuncSetAttribute(region_attention_store_kernel<D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes)
+                  : cudaFuncSetAttribute(region_attention_tc_kernel<D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+        if (e != cudaSuccess) return REGIONE_CUDA_ERROR;
         __atomic_store_n(&configured[dev], 1, __ATOMIC_RELEASE);
     }
-    if (launch_overlapped(region_attention_tc_kernel<D, STORE>, dim3(grid), dim3(kAttnThreads),
-                          Cfg::kSmemBytes, st, maps[0], maps[1], maps[2], maps[3], maps[4],
-                          prm) != cudaSuccess)
-        return REGIONE_CUDA_ERROR;
-    return REGIONE_OK;
+    cudaError_t e;
+    if constexpr (STORE)
+        e = launch_overlapped(region_attention_store_kernel<D>, dim3(grid), dim3(kAttnThreads),
+                              Cfg::kSmemBytes, st, maps[0], maps[1], maps[2], maps[3], maps[4], prm, sp);
+    else
+        e = launch_overlapped(region_attention_tc_kernel<D>, dim3(grid), dim3(kAttnThreads),
+                              Cfg::kSmemBytes, st, maps[0], maps[1], maps[2], maps[3], maps[4], prm);
+    return e == cudaSuccess ? REGIONE_OK : REGIONE_CUDA_ERROR;
 }
 
 template <int D>
-static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, int grid, cudaStream_t st) {
-    const int rc = prm.keep_rows != nullptr ? launch_main<D, true>(maps, prm, grid, st)
-                                            : launch_main<D, false>(maps, prm, grid, st);
+static int launch_tc(const CUtensorMap* maps, const AttnParams& prm, const StoreParams* sp, int grid,
+                     cudaStream_t st) {
+    const StoreParams none = {};
+    const int rc = sp != nullptr ? launch_main<D, true>(maps, prm, *sp, grid, st)
+                                 : launch_main<D, false>(maps, prm, none, grid, st);
     if (rc != REGIONE_OK) return rc;
     // the merge kernel may become resident while the attention kernel drains (it waits for that
     // kernel's completion before it reads a slot)
@@ -1237,18 +1270,19 @@ int launch_region_attention_tc(const uint16_t* q, const uint16_t* k_fresh, const
     prm.out_rows = out_rows;
     prm.out_cap = out_rows != nullptr ? out_cap : Nq_cap;
     prm.timeout_cycles = kTimeoutCycles;
-    prm.keep_rows = store != nullptr ? store->keep_rows : nullptr;
-    prm.n_keep = store != nullptr ? store->n_keep : nullptr;
-    prm.store_cap = store != nullptr ? store->cap : 0;
-    prm.k_store = store != nullptr ? store->k_cache : nullptr;
-    prm.v_store = store != nullptr ? store->v_cache : nullptr;
+    StoreParams sp = {};
+    if (store != nullptr) {
+        sp.keep_rows = store->keep_rows; sp.n_keep = store->n_keep; sp.store_cap = store->cap;
+        sp.k_store = store->k_cache; sp.v_store = store->v_cache;
+    }
     const size_t rows = slot_rows(lp, B, H);
     prm.part_o = reinterpret_cast<float*>(workspace);
     uint8_t* const ws = reinterpret_cast<uint8_t*>(workspace);
     const size_t off_ml = (rows * D * sizeof(float) + 255) & ~(size_t)255;
     prm.part_ml = reinterpret_cast<float2*>(ws + off_ml);
     prm.cut = reinterpret_cast<CutItem*>(ws + off_ml + ((rows * sizeof(float2) + 255) & ~(size_t)255));
-    return D == 64 ? launch_tc<64>(maps, prm, lp.grid, st) : launch_tc<128>(maps, prm, lp.grid, st);
+    const StoreParams* spp = store != nullptr ? &sp : nullptr;
+    return D == 64 ? launch_tc<64>(maps, prm, spp, lp.grid, st) : launch_tc<128>(maps, prm, spp, lp.grid, st);
 }
 
 // ---- variant with library-owned scratch -----------------------------------------------------
