@@ -91,17 +91,21 @@ struct AttnCtrl {
     uint64_t s_full[2];         // [query tile]
     uint64_t p_full[2][2];      // [query tile][chunk of 64 keys]
     uint64_t o_final[2];        // completes once, after the tile's last P*V product
-    uint64_t turn[2];           // turn[t]: the other query tile has finished a tile's exponentials
+    uint64_t pv_done[2];        // [query tile] completes after every key tile's last product: P may be
+                                // overwritten and O rescaled
+    uint64_t s_free;            // the shared S buffer has been read by the softmax warps it was computed for
     uint64_t half_done;         // lone query tile: the odd key tiles' (max, sum) are in shared memory
     uint32_t tmem_base;
     int abort_flag;
 };
 
 // The barriers of AttnCtrl as one array starting at q_full.
-constexpr int kBarKvEmpty = 9, kBarSFull = 17, kBarPFull = 19, kBarOFinal = 23, kBarTurn = 25, kNumBarriers = 28;
+constexpr int kBarKvEmpty = 9, kBarSFull = 17, kBarPFull = 19, kBarOFinal = 23, kBarPvDone = 25, kBarSFree = 27,
+              kBarHalfDone = 28, kNumBarriers = 29;
 static_assert(offsetof(AttnCtrl, kv_empty) == kBarKvEmpty * 8 && offsetof(AttnCtrl, s_full) == kBarSFull * 8 &&
               offsetof(AttnCtrl, p_full) == kBarPFull * 8 && offsetof(AttnCtrl, o_final) == kBarOFinal * 8 &&
-              offsetof(AttnCtrl, turn) == kBarTurn * 8 && offsetof(AttnCtrl, tmem_base) == kNumBarriers * 8,
+              offsetof(AttnCtrl, pv_done) == kBarPvDone * 8 && offsetof(AttnCtrl, s_free) == kBarSFree * 8 &&
+              offsetof(AttnCtrl, half_done) == kBarHalfDone * 8 && offsetof(AttnCtrl, tmem_base) == kNumBarriers * 8,
               "barrier layout");
 
 // What share c tells the merge kernel: the item that the boundary between shares c - 1 and c
@@ -436,9 +440,10 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
     // a lone tile's ring starts at the idle second query tile and runs over the extra stage: two
     // stages more, because its two halves consume K/V tiles at twice the rate per chain
     const int n_stages = split ? kStages + 2 : kStages;
-    // cache refresh: the first query pair of every (request, head) also writes the retained rows of
-    // the key tiles it walks, so every (request, head, key tile) is written exactly once
-    const bool store_item = STORE && it.qp == 0 && n_tiles > 0;
+    // cache refresh: every item walks all key tiles of its (request, head); key tile j is written to
+    // the cache by the item of query pair j mod np, so every (request, head, key tile) is written
+    // exactly once and the copies are spread evenly over the thread blocks
+    const bool store_item = STORE && n_tiles > 0;
     const uint32_t ring = split ? sQ + kTileBytes : sKV;
     uint8_t* const ring_gen = smem_gen + (split ? 1 : 2) * kTileBytes;
 
@@ -447,7 +452,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         const int i = threadIdx.x;
         int count = 1;                                               // q_full, kv_full, s_full, o_final
         if (i >= kBarKvEmpty && i < kBarSFull) count = (split ? 1 : ntq) + (store_item ? 1 : 0);   // commits per stage (+ the cache writer)
-        else if ((i >= kBarPFull && i < kBarOFinal) || i >= kBarTurn) count = kBM / 32;   // one arrival per warp
+        else if ((i >= kBarPFull && i < kBarOFinal) || i >= kBarSFree) count = kBM / 32;   // one arrival per warp
         ptx::mbar_init(ptx::smem_addr(&ctrl->q_full + i), count);
         ptx::fence_barrier_init();
     }
@@ -476,86 +481,89 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
 
     if constexpr (!SOFTMAX_WG) {
     if (warp == 8) {
-        // ================= TMA producer =================
-        if (lane == 0 && n_tiles > 0) {
-            ptx::prefetch_tensormap(&tm_q);
-            ptx::prefetch_tensormap(j_first < nt_c ? &tm_kc : &tm_kf);
-            ptx::prefetch_tensormap(j_first < nt_c ? &tm_vc : &tm_vf);
-            const uint32_t qbar = ptx::smem_addr(&ctrl->q_full);
-            ptx::mbar_arrive_expect_tx(qbar, ntq * kTileBytes);
-            for (int t = 0; t < ntq; ++t)
-                for (int hf = 0; hf < Cfg::kHalves; ++hf)
-                    ptx::tma_load_4d(sQ + t * kTileBytes + hf * kHalfBytes, &tm_q, qbar, hf * 64, h,
-                                     q0 + t * kBM, b);
-            bool ok = true;
-            for (int i = 0; i < 2 * n_tiles && ok; ++i) {
-                const int j = i >> 1, is_v = i & 1;
-                const int stage = i % n_stages, use = i / n_stages;
-                if (use > 0)
-                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_empty[stage]), (use - 1) & 1, abort_flag,
-                                  p.dev_status, p.timeout_cycles);
-                if (!ok) break;
-                bool cached; int row0, valid;
-                tile_seg(j, cached, row0, valid);
-                const CUtensorMap* map = cached ? (is_v ? &tm_vc : &tm_kc) : (is_v ? &tm_vf : &tm_kf);
-                const uint32_t bar = ptx::smem_addr(&ctrl->kv_full[stage]);
-                ptx::mbar_arrive_expect_tx(bar, kTileBytes);
-                for (int hf = 0; hf < Cfg::kHalves; ++hf)
-                    ptx::tma_load_4d(ring + stage * kTileBytes + hf * kHalfBytes, map, bar, hf * 64, h,
-                                     row0, b);
+        // ================= TMA producer (and, in the cache-refreshing kernel, the cache writer) =================
+        if (n_tiles > 0) {
+            if (lane == 0) {
+                ptx::prefetch_tensormap(&tm_q);
+                ptx::prefetch_tensormap(j_first < nt_c ? &tm_kc : &tm_kf);
+                ptx::prefetch_tensormap(j_first < nt_c ? &tm_vc : &tm_vf);
+                const uint32_t qbar = ptx::smem_addr(&ctrl->q_full);
+                ptx::mbar_arrive_expect_tx(qbar, ntq * kTileBytes);
+                for (int t = 0; t < ntq; ++t)
+                    for (int hf = 0; hf < Cfg::kHalves; ++hf)
+                        ptx::tma_load_4d(sQ + t * kTileBytes + hf * kHalfBytes, &tm_q, qbar, hf * 64, h,
+                                         q0 + t * kBM, b);
             }
-        }
-    } else if (STORE && warp == 11) {
-        // ================= cache writer (full step that refreshes the RIKV cache) =================
-        if (store_item) {
+            // ---- cache writer state (whole warp; used by the cache-refreshing kernel only) ----
+            // The retained rows of every K / V tile this segment stages are copied from shared memory
+            // to their slots in the cache, two ring items behind the loads (an item has landed by
+            // then), before its stage is given back.
             constexpr int kCpr = D / 8;                 // 16-byte chunks per row of one head
             constexpr int kRowsPer = 32 / kCpr;         // rows a warp instruction moves
-            const int32_t* keep = sp.keep_rows + (size_t)b * sp.store_cap;
-            int nk = sp.n_keep[b];
-            if (nk < 0 || nk > sp.store_cap) {
-                record_status(p.dev_status, REGIONE_DEV_BOUNDS);
-                nk = max(0, min(nk, sp.store_cap));
+            constexpr int kLag = 2;
+            const int32_t* keep = nullptr;
+            int nk = 0, lo = 0, cnt = 0;
+            bool mine = false;                          // the key tile being written belongs to this item
+            int r[kBN / 32];
+            if (STORE && store_item) {
+                keep = sp.keep_rows + (size_t)b * sp.store_cap;
+                nk = sp.n_keep[b];
+                if (nk < 0 || nk > sp.store_cap) {
+                    record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+                    nk = max(0, min(nk, sp.store_cap));
+                }
             }
-            // first retained row at or behind this segment's first key row: 32-ary search, one
+            // number of retained rows below `row_first` (the list is ascending): 32-ary search, one
             // coalesced probe per level
-            const int row_first = j_first * kBN;        // (a full step has no cached segment)
-            int lo = 0, len = nk;
-            while (len > 0) {
-                const int step = (len + 31) / 32;
-                const int at = lo + min(lane * step, len - 1);
-                const bool below = (lane * step < len) && keep[at] < row_first;
-                const int nb = __popc(__ballot_sync(0xffffffffu, below));   // probes below the target
-                // the answer lies behind probe nb - 1 and at or before probe nb
-                const int new_lo = nb == 0 ? lo : lo + (nb - 1) * step + 1;
-                const int new_hi = nb == 0 ? lo : min(lo + nb * step, lo + len);
-                len = (step == 1) ? 0 : new_hi - new_lo;
-                lo = (step == 1) ? lo + nb : new_lo;
-            }
-            bool ok = true;
-            for (int jl = 0; jl < n_tiles && ok; ++jl) {
+            auto rows_below = [&](int row_first) {
+                int at0 = 0, len = nk;
+                while (len > 0) {
+                    const int step = (len + 31) / 32;
+                    const int at = at0 + min(lane * step, len - 1);
+                    const bool below = (lane * step < len) && keep[at] < row_first;
+                    const int nb = __popc(__ballot_sync(0xffffffffu, below));   // probes below the target
+                    // the answer lies behind probe nb - 1 and at or before probe nb
+                    const int new_lo = nb == 0 ? at0 : at0 + (nb - 1) * step + 1;
+                    const int new_hi = nb == 0 ? at0 : min(at0 + nb * step, at0 + len);
+                    len = (step == 1) ? 0 : new_hi - new_lo;
+                    at0 = (step == 1) ? at0 + nb : new_lo;
+                }
+                return at0;
+            };
+            // copies ring item x (K of key tile x / 2, or V) to the cache if that tile is this item's to
+            // write, and releases its stage
+            auto write_item = [&](int x) -> bool {
+                const int jl = x >> 1, is_v = x & 1, stage = x % n_stages;
                 bool cached; int row0, valid;
                 tile_seg(jl, cached, row0, valid);
-                // retained rows of this tile: at most kBN consecutive entries of the ascending list
-                int r[kBN / 32];
-                int cnt = 0;                            // length of the run of entries inside this tile
-                bool run_open = true;
+                if (!is_v) {
+                    mine = (j_first + jl) % it.r.np == it.qp;
+                    if (mine) {
+                        // retained rows of this tile: at most kBN consecutive entries of the ascending list
+                        lo = rows_below(row0);
+                        cnt = 0;                        // length of the run of entries inside this tile
+                        bool run_open = true;
 #pragma unroll
-                for (int k = 0; k < kBN / 32; ++k) {
-                    const int i = lo + k * 32 + lane;
-                    r[k] = i < nk ? keep[i] - row0 : kBN;
-                    if (r[k] < 0) {                     // the list is not ascending
-                        record_status(p.dev_status, REGIONE_DEV_BOUNDS);
-                        r[k] = kBN;
+                        for (int k = 0; k < kBN / 32; ++k) {
+                            const int i = lo + k * 32 + lane;
+                            r[k] = i < nk ? keep[i] - row0 : kBN;
+                            if (r[k] < 0) {             // the list is not ascending
+                                record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+                                r[k] = kBN;
+                            }
+                            const uint32_t inside = __ballot_sync(0xffffffffu, r[k] < valid);
+                            if (run_open) cnt += inside == 0xffffffffu ? 32 : __ffs(~inside) - 1;
+                            run_open = run_open && inside == 0xffffffffu;
+                        }
+                        // entries left over behind the last key tile name rows that do not exist
+                        if (j_first + jl == it.r.nt - 1 && lo + cnt < nk)
+                            record_status(p.dev_status, REGIONE_DEV_BOUNDS);
                     }
-                    const uint32_t inside = __ballot_sync(0xffffffffu, r[k] < valid);
-                    if (run_open) cnt += inside == 0xffffffffu ? 32 : __ffs(~inside) - 1;
-                    run_open = run_open && inside == 0xffffffffu;
                 }
-                for (int is_v = 0; is_v < 2 && ok; ++is_v) {
-                    const int i_ring = 2 * jl + is_v, stage = i_ring % n_stages;
-                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[stage]), (i_ring / n_stages) & 1, abort_flag,
-                                  p.dev_status, p.timeout_cycles);
-                    if (!ok) break;
+                if (mine) {
+                    if (!wait_bar(ptx::smem_addr(&ctrl->kv_full[stage]), (x / n_stages) & 1, abort_flag,
+                                  p.dev_status, p.timeout_cycles))
+                        return false;
                     const uint8_t* tile = ring_gen + stage * kTileBytes;
                     uint16_t* dst_base = (is_v ? sp.v_store : sp.k_store) +
                                          (((size_t)b * sp.store_cap + lo) * p.H + h) * D;
@@ -563,80 +571,123 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
 #pragma unroll
                     for (int k = 0; k < kBN / 32; ++k) {
                         if (k * 32 >= cnt) break;                       // (uniform)
-#pragma unroll 2
-                        for (int e1 = 0; e1 < 32; e1 += kRowsPer) {
-                            const int el = e1 + lane / kCpr;            // entry of the tile's run: k * 32 + el
-                            const int rr = __shfl_sync(0xffffffffu, r[k], el);
-                            if (k * 32 + el < cnt) {
-                                const uint4 x = *reinterpret_cast<const uint4*>(
-                                    tile + (q >> 3) * kHalfBytes + rr * 128 + (((q & 7) ^ (rr & 7)) << 4));
-                                *reinterpret_cast<uint4*>(dst_base + (size_t)(k * 32 + el) * p.H * D + q * 8) = x;
+#pragma unroll 1
+                        for (int e0 = 0; e0 < 32; e0 += 4 * kRowsPer) {
+                            // four warp-wide moves at a time: all loads are issued before the first store
+                            uint4 x4[4];
+                            int el[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                el[u] = e0 + u * kRowsPer + lane / kCpr;    // entry of the tile's run: k * 32 + el
+                                const int rr = __shfl_sync(0xffffffffu, r[k], el[u]);
+                                if (k * 32 + el[u] < cnt)
+                                    x4[u] = *reinterpret_cast<const uint4*>(
+                                        tile + (q >> 3) * kHalfBytes + rr * 128 + (((q & 7) ^ (rr & 7)) << 4));
                             }
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                if (k * 32 + el[u] < cnt)
+                                    *reinterpret_cast<uint4*>(dst_base + (size_t)(k * 32 + el[u]) * p.H * D + q * 8) = x4[u];
                         }
                     }
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->kv_empty[stage]));
                 }
-                lo += cnt;
-                // entries left over behind the item's last key tile name rows that do not exist
-                if (j_first + jl == it.r.nt - 1 && lo < nk) record_status(p.dev_status, REGIONE_DEV_BOUNDS);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->kv_empty[stage]));
+                return true;
+            };
+            bool ok = true;
+            const int n_items = 2 * n_tiles;
+            for (int i = 0; i < n_items + (STORE && store_item ? kLag : 0) && ok; ++i) {
+                if (STORE && store_item && i >= kLag) ok = write_item(i - kLag);
+                if (i < n_items && ok) {
+                    if (lane == 0) {
+                        const int j = i >> 1, is_v = i & 1;
+                        const int stage = i % n_stages, use = i / n_stages;
+                        if (use > 0)
+                            ok = wait_bar(ptx::smem_addr(&ctrl->kv_empty[stage]), (use - 1) & 1, abort_flag,
+                                          p.dev_status, p.timeout_cycles);
+                        if (ok) {
+                            bool cached; int row0, valid;
+                            tile_seg(j, cached, row0, valid);
+                            const CUtensorMap* map = cached ? (is_v ? &tm_vc : &tm_kc) : (is_v ? &tm_vf : &tm_kf);
+                            const uint32_t bar = ptx::smem_addr(&ctrl->kv_full[stage]);
+                            ptx::mbar_arrive_expect_tx(bar, kTileBytes);
+                            for (int hf = 0; hf < Cfg::kHalves; ++hf)
+                                ptx::tma_load_4d(ring + stage * kTileBytes + hf * kHalfBytes, map, bar, hf * 64, h,
+                                                 row0, b);
+                        }
+                    }
+                    if (STORE) ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;     // (the writer's lanes follow lane 0)
+                }
+            }
+        }
+    } else if (warp == 11) {
+        // ================= issuer of the S products of both query tiles =================
+        // S = Q_t K_j^T goes to ONE staging buffer in tensor memory that the two query tiles share:
+        // a product is issued as soon as its K tile has landed and the buffer's previous contents
+        // have been read into registers by the softmax warps they were computed for.  It does not
+        // have to wait for the P*V products of its own tile, which read P from a place of their own.
+        if (n_tiles > 0) {
+            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
+            constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
+            const uint32_t k_lo = ptx::smem_desc_lo(ring, 16);
+            bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status, p.timeout_cycles);
+            int n_issued = 0;                                   // products so far = uses of the staging buffer
+            for (int jl = 0; jl < n_tiles && ok; ++jl) {
+                const int ik = 2 * jl, sk = ik % n_stages;
+                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / n_stages) & 1, abort_flag,
+                              p.dev_status, p.timeout_cycles);
+                // the roles this key tile feeds: both query tiles, or one half of a lone query tile
+                const int t_first = split ? (jl & 1) : 0, t_last = split ? (jl & 1) : ntq - 1;
+                for (int t = t_first; t <= t_last && ok; ++t) {
+                    if (n_issued > 0)
+                        ok = wait_bar(ptx::smem_addr(&ctrl->s_free), (n_issued - 1) & 1, abort_flag,
+                                      p.dev_status, p.timeout_cycles);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    if (ptx::elect_one()) {
+                        const uint32_t q_lo = ptx::smem_desc_lo(sQ + (split ? 0 : t) * kTileBytes, 16);
+                        const uint32_t b0 = k_lo + ((sk * kTileBytes) >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                            ptx::mma_ss(tmem, ptx::smem_desc_join(q_lo + off, hi_k),
+                                        ptx::smem_desc_join(b0 + off, hi_k), idesc_s, kk > 0);
+                        }
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
+                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk]));
+                    }
+                    __syncwarp();
+                    ++n_issued;
+                }
             }
         }
     } else if (warp == 9 || warp == 10) {
-        // ================= MMA issuers: warp 9 for query tile 0, warp 10 for query tile 1 ========
+        // ================= issuers of the P*V products: warp 9 for query tile 0, warp 10 for query tile 1 ========
         // Each whole warp walks its loop and waits on the barriers; one elected lane issues.
         const int t = warp - 9;
         if (t < lanes && n_tiles > 0) {
             const int n_my = role_tiles(t);
-            constexpr uint32_t idesc_s = ptx::idesc_bf16_f32(kBM, kBN, false);
             constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kBM, D, true);
-            constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-row groups 1024 B apart
-            // K-major operands (Q, K): 128-byte swizzle, LBO unused; V is MN-major: 64-column
-            // boxes kHalfBytes apart (LBO), 8-key groups 1024 B apart (SBO).
-            const uint32_t q_lo = ptx::smem_desc_lo(sQ + (split ? 0 : t) * kTileBytes, 16);
-            const uint32_t k_lo = ptx::smem_desc_lo(ring, 16);
+            constexpr uint32_t hi_k = ptx::smem_desc_hi_sw128(1024);   // 8-key groups 1024 B apart
+            // V is MN-major: 64-column boxes kHalfBytes apart (LBO), 8-key groups 1024 B apart (SBO)
             const uint32_t v_lo = ptx::smem_desc_lo(ring, kHalfBytes);
-            const uint32_t tSt = tmem + t * kBN, tOt = tmem + 256 + t * D;
-            // S_t = Q_t K^T
-            auto issue_s = [&](int stage) {
-                const uint32_t b0 = k_lo + ((stage * kTileBytes) >> 4);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
-                    ptx::mma_ss(tSt, ptx::smem_desc_join(q_lo + off, hi_k),
-                                ptx::smem_desc_join(b0 + off, hi_k), idesc_s, kk > 0);
-                }
-            };
+            const uint32_t tPt = tmem + kBN + t * (kBN / 2), tOt = tmem + 256 + t * D;
             // O_t (+)= P_t[chunk] V[64 chunk .. 64 chunk + 64) : A from tensor memory (bf16 pairs,
             // 8 columns per 16 keys)
             auto issue_pv = [&](int stage, int chunk, bool accumulate) {
                 const uint32_t b0 = v_lo + ((stage * kTileBytes + chunk * (kBH / 16) * 2048) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < kBH / 16; ++kk)
-                    ptx::mma_ts(tOt, tSt + chunk * (kBH / 2) + kk * 8,
+                    ptx::mma_ts(tOt, tPt + chunk * (kBH / 2) + kk * 8,
                                 ptx::smem_desc_join(b0 + ((kk * 2048) >> 4), hi_k), idesc_pv,
                                 (accumulate || kk > 0) ? 1u : 0u);
             };
-            bool ok = wait_bar(ptx::smem_addr(&ctrl->q_full), 0, abort_flag, p.dev_status, p.timeout_cycles);
-            if (ok) {
-                const int ik0 = 2 * role_tile(t, 0), sk0 = ik0 % n_stages;
-                ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk0]), (ik0 / n_stages) & 1, abort_flag,
-                              p.dev_status, p.timeout_cycles);
-                if (ok) {
-                    ptx::tc_fence_after_sync();
-                    if (ptx::elect_one()) {
-                        issue_s(sk0);
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk0]));
-                    }
-                    __syncwarp();
-                }
-            }
+            bool ok = true;
             int nb = 0;                                     // second chunks seen so far
             for (int j = 0; j < n_my && ok; ++j) {
                 const int jl = role_tile(t, j);
-                const int iv = 2 * jl + 1, ik = 2 * role_tile(t, j + 1);
-                const int sv = iv % n_stages, sk = ik % n_stages;
+                const int iv = 2 * jl + 1, sv = iv % n_stages;
                 const bool more = (j + 1 < n_my);
                 const int chunks = tile_chunks(jl);
                 ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sv]), (iv / n_stages) & 1, abort_flag,
@@ -649,26 +700,17 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                     ptx::tc_fence_after_sync();
                     if (ptx::elect_one()) issue_pv(sv, 0, j > 0);
                     __syncwarp();
-                }
-                if (more)
-                    ok = wait_bar(ptx::smem_addr(&ctrl->kv_full[sk]), (ik / n_stages) & 1, abort_flag,
-                                  p.dev_status, p.timeout_cycles);
-                if (ok && chunks == 2) {
                     ok = wait_bar(ptx::smem_addr(&ctrl->p_full[t][1]), nb & 1, abort_flag,
                                   p.dev_status, p.timeout_cycles);
                     ++nb;
+                    if (!ok) break;
                 }
-                if (!ok) break;
                 ptx::tc_fence_after_sync();
                 if (ptx::elect_one()) {
                     issue_pv(sv, chunks - 1, j > 0 || chunks == 2);
+                    ptx::mma_commit(ptx::smem_addr(&ctrl->pv_done[t]));
                     if (!more) ptx::mma_commit(ptx::smem_addr(&ctrl->o_final[t]));
                     ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sv]));
-                    if (more) {
-                        issue_s(sk);
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->s_full[t]));
-                        ptx::mma_commit(ptx::smem_addr(&ctrl->kv_empty[sk]));
-                    }
                 }
                 __syncwarp();
             }
@@ -679,7 +721,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
         const int t = warp >> 2;
         const int row = ((warp & 3) << 5) + lane;                  // row of the query tile
         const uint32_t lane_sel = (uint32_t)((warp & 3) << 5) << 16;
-        const uint32_t tS = tmem + lane_sel + t * kBN;
+        const uint32_t tS = tmem + lane_sel;                       // the S staging buffer both tiles share
+        const uint32_t tP = tmem + lane_sel + kBN + t * (kBN / 2); // this tile's probabilities (bf16 pairs)
         const uint32_t tO = tmem + lane_sel + 256 + t * D;
         const float c = p.scale_log2e;
         float m = -INFINITY, l = 0.f;
@@ -693,25 +736,36 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             ok = wait_bar(ptx::smem_addr(&ctrl->s_full[t]), j & 1, abort_flag, p.dev_status, p.timeout_cycles);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            // (P_t V_{j-1} has completed here: S_t(j) was issued after it by the same thread and
-            // tcgen05.mma executes in issue order, so O_t may be rescaled and P_t overwritten)
             uint32_t s[kBN];
             ptx::tmem_ld32(tS, s);
             ptx::tmem_ld32(tS + 32, s + 32);
-            ptx::tmem_wait_ld();
-            float mt;
             if (chunks == 2) {
                 ptx::tmem_ld32(tS + 64, s + 64);
                 ptx::tmem_ld32(tS + 96, s + 96);
-                mt = chunk_max(s);
-                ptx::tmem_wait_ld();
+            }
+            ptx::tmem_wait_ld();
+            // the logits are in registers: the staging buffer may take the next product (of the other
+            // query tile, or of this tile's next key tile)
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->s_free));
+            float mt;
+            if (chunks == 2) {
                 if (valid < kBN) mask_dead_keys(s + kBH, valid - kBH);
-                mt = fmaxf(mt, chunk_max(s + kBH));
+                mt = fmaxf(chunk_max(s), chunk_max(s + kBH));
             } else {
                 if (valid < kBH) mask_dead_keys(s, valid);
                 mt = chunk_max(s);
             }
             mt *= c;
+            // P_t and O_t belong to the products of the key tile before this one until they have
+            // completed (they run in the shadow of this tile's wait for S and of its row maximum)
+            if (j > 0) {
+                ok = wait_bar(ptx::smem_addr(&ctrl->pv_done[t]), (j - 1) & 1, abort_flag, p.dev_status,
+                              p.timeout_cycles);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+            }
             if (j == 0) {
                 m = mt;
             } else if (__any_sync(0xffffffffu, mt > m + 8.f)) {
@@ -729,20 +783,8 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
                 l *= alpha;
                 m = m_new;
             }
-            // The two query tiles take turns on the special-function unit: tile 1 computes the
-            // exponentials of key tile j after tile 0 has finished its own, tile 0 those of key
-            // tile j + 1 after tile 1 has finished j.  Run alone they take half as long, which
-            // shortens each tile's chain S -> softmax -> P*V -> next S; the other tile's loads,
-            // maxima and products fall into the gap.
-            if (lanes == 2 && (t == 1 || j > 0)) {
-                ok = wait_bar(ptx::smem_addr(&ctrl->turn[t]), (j - 1 + t) & 1, abort_flag,
-                              p.dev_status, p.timeout_cycles);
-                if (!ok) break;
-            }
             // first chunk of probabilities (keys 0..63 of the tile)
-            l += chunk_probabilities(tS, s, c, m);
-            if (chunks == 1 && lanes == 2 && lane == 0)
-                ptx::mbar_arrive(ptx::smem_addr(&ctrl->turn[t ^ 1]));
+            l += chunk_probabilities(tP, s, c, m);
             ptx::tmem_wait_st();
             if (valid < kBN) {
                 // last tile of a segment: zero the V rows behind the live prefix (0 * NaN = NaN)
@@ -765,8 +807,7 @@ __device__ __forceinline__ void run_share(const CUtensorMap* tm_q_, const CUtens
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->p_full[t][0]));
             if (chunks == 2) {
                 // second chunk (keys 64..127) while the first chunk's product runs
-                l += chunk_probabilities(tS + kBH / 2, s + kBH, c, m);
-                if (lanes == 2 && lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctrl->turn[t ^ 1]));
+                l += chunk_probabilities(tP + kBH / 2, s + kBH, c, m);
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
