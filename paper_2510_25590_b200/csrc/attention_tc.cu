@@ -8,27 +8,34 @@
 //   warps 4-7  the same for query tile 1
 //   warp  8    TMA producer: Q once, then K_j, V_j tiles (128 keys) through a ring
 //              of shared-memory stages; the cached segment and the fresh segment
-//              are two tensor maps walked one after the other
-//   warps 9,10 tcgen05.mma issuers, one per query tile (the whole warp walks the
-//              loop, one elected lane issues); warp 9 owns the tensor-memory allocation
-//   warp  11   fills the third warpgroup so that registers can be moved from it to the
-//              softmax warpgroups with setmaxnreg; idle, except in the full step that
-//              refreshes the Region-Instruction KV cache: there it copies the retained rows of
-//              every staged K / V tile from shared memory to their places in the cache
+//              are two tensor maps walked one after the other.  In the full step that
+//              refreshes the Region-Instruction KV cache the whole warp also copies the
+//              retained rows of the staged K / V tiles from shared memory to the cache
+//   warps 9,10 issuers of the O_t += P_t V_j products, one per query tile (the whole
+//              warp walks the loop, one elected lane issues); warp 9 owns the
+//              tensor-memory allocation
+//   warp  11   issuer of the S = Q_t K_j^T products of both query tiles
+//   (warps 8-11 form the third warpgroup; it gives registers up to the softmax
+//   warpgroups with setmaxnreg)
 //
-// Tensor memory (512 columns): S0 | S1 | O0 | O1.  S_t = Q_t K_j^T (fp32, 128
-// columns) is read back by the softmax warps of tile t, the probabilities are
-// written over it as packed bf16 (P aliases the first 64 columns of S) in two
-// chunks of 64 keys, and O_t += P_t V_j runs straight from tensor memory: the
-// product of the first chunk is issued while the exponentials of the second
-// are still being computed.  Each query tile has its own issuer warp, so the
-// dependency chain of a tile (S -> softmax -> P*V -> next S) only stalls that
-// tile; the other tile's products fill the tensor pipe meanwhile.  The two
-// tiles take turns on the special-function unit (exp2), which keeps them out
-// of phase.  A pair with a single live query tile does not leave the second
-// tile's warps idle: they run the same query tile against the odd key tiles of
-// the segment (own accumulator, maximum and sum in tensor memory / registers),
-// the first tile's warps take the even ones, and the epilogue merges the halves.
+// Tensor memory (512 columns): S | P0 | P1 | O0 | O1 = 128 + 64 + 64 + 128 + 128.
+// There is ONE S buffer (fp32, 128 logits per row), a staging place that the two
+// query tiles share: a product lands there, the softmax warps of its tile read their
+// row into registers and give the buffer back at once, and the next product (the other
+// tile's, or the same tile's next key tile) may follow while the exponentials are
+// still being computed.  The probabilities go to the tile's own P region as packed
+// bf16, in two chunks of 64 keys, and O_t += P_t V_j runs straight from tensor memory:
+// the product of the first chunk is issued while the exponentials of the second are
+// computed.  Because P does not live in the S buffer, S_t(j+1) never waits for the
+// products P_t(j) V_j: the dependency chain of a tile is  S ready -> row maximum ->
+// exponentials -> (S of the next key tile is already there),  with both kinds of
+// product off it.  What a tile must wait for before it overwrites P_t or rescales O_t
+// is the completion of its previous key tile's products (a barrier of their own), and
+// that has long happened by then.  The two tiles run their exponentials whenever they
+// are ready; nothing sequences them.  A pair with a single live query tile does not
+// leave the second tile's warps idle: they run the same query tile against the odd key
+// tiles of the segment (own accumulator, maximum and sum), the first tile's warps take
+// the even ones, and the epilogue merges the halves.
 //
 // Online softmax in the exp2 domain; O is rescaled in tensor memory only when
 // a row maximum grows by more than 2^8.  Keys past a segment's live count are
