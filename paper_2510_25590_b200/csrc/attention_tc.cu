@@ -157,7 +157,7 @@ struct StoreParams {
 // tile kTickSingle (its even and odd key tiles run side by side on the two tile roles, so it costs
 // half as much), and every item starts with kTickStart ticks that stand for the
 // drain of the previous segment and the fill of the new one (measured on the kernel).
-constexpr int kTickPair = 8, kTickSingle = 4, kTickStart = 28;
+constexpr int kTickPair = 8, kTickSingle = 4, kTickStart = 36;
 
 struct ReqShape {
     int nq, nf, nc;      // clamped counts
