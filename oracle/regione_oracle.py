@@ -51,7 +51,7 @@ def token_score(x0_hat, ref, metric):
     """One score per token, reduced over that token's channels.
 
     metric COSINE: cosine similarity between the estimate and the instruction
-    (reference) latent "along the token dimension" (Adaptive Region Partition
+    (reference) latent, one value per token (Adaptive Region Partition
     paragraph).  A zero denominator is clamped at 1e-12.
     metric L2: Euclidean distance over the channels (not squared, not averaged).
     """
@@ -67,7 +67,7 @@ def token_score(x0_hat, ref, metric):
 
 
 def edit_mask(score, metric, threshold):
-    """mask = 1 (edited) unless the token is "sufficiently similar" to the reference.
+    """mask = 1 (edited) unless the token is similar enough to the reference.
 
     Cosine: the paper calls a token unedited iff similarity > eta (strict), so
     it is edited iff s <= eta.  L2: edited iff distance > tau, unedited iff
@@ -164,8 +164,8 @@ def _dilate3(m):
 def open_close(mask, grid):
     """Opening (erode, dilate) then closing (dilate, erode) of the edited mask.
 
-    The Adaptive Region Partition paragraph applies "morphological opening and
-    closing"; the structuring element is not given: a 3x3 square on the
+    The Adaptive Region Partition paragraph cleans the mask with a morphological
+    opening and closing; the structuring element is not given: a 3x3 square on the
     rows x cols token grid is used, out-of-grid neighbours ignored.
     """
     m = np.asarray(mask).astype(np.uint8).reshape(grid)
@@ -211,8 +211,8 @@ def scatter(dst, src, idx, n):
 def rikv_store(k_full, v_full, keep_rows, n_keep):
     """K^C, V^C: the retained rows of the last full step's K and V.
 
-    Stabilization Stage paragraph ("save the Key and Value in each attention
-    layer"), refreshed at forced steps.  k_full, v_full: [B, n_full, H, D];
+    Stabilization Stage paragraph (K and V of every attention layer are kept at
+    the last full step), refreshed at forced steps.  k_full, v_full: [B, n_full, H, D];
     keep_rows [B, cap]; returns (k_cache, v_cache) [B, cap, H, D], NaN past n_keep[b].
     """
     return gather(k_full, keep_rows, n_keep), gather(v_full, keep_rows, n_keep)
