@@ -200,6 +200,34 @@ int regione_rikv_store(const regione_bf16* k_full, const regione_bf16* v_full,
                        int32_t* dev_status, void* stream);
 
 /*
+ * 8-bit variant of the Region-Instruction KV cache.  (Sec. 4 "Stabilization Stage" keeps K and V of
+ * every attention layer from one full step to the next forced one; the paper keeps them in the
+ * model's precision, so this storage format has no counterpart there.)  regione_rikv_store_e4m3 is
+ * regione_rikv_store with the retained rows written as 8-bit floating point E4M3 (1 sign, 4 exponent,
+ * 3 mantissa bits, bias 7, largest finite value 448, no infinities) and one power-of-two scale per
+ * (row, head): half the bytes per cached layer.  regione_rikv_load_e4m3 widens such a cache back
+ * to bf16 in front of a region step's attention:
+ *     s = 2^k, k the smallest integer with max_d |x[b,row,h,d]| / 2^k <= 448   (k = 0 for an all-zero
+ *         row and head; k >= -100)
+ *     code = nearest E4M3 value of x / s, ties to the even mantissa
+ *     k_cache[b,j,h,d] = value(code) * s        (exact in bf16: no second rounding)
+ * k_full, v_full [B, N_full, H, D] bf16; keep_rows dev int32 [B, Nc_cap]; n_keep dev int32 [B];
+ * k_q, v_q dev u8 [B, Nc_cap, H, D]; k_scale, v_scale dev f32 [B, Nc_cap, H];
+ * k_cache, v_cache dev bf16 [B, Nc_cap, H, D].  Rows past n_keep[b] are left untouched by both.
+ * D must be 64 or 128.  NaN elements are not preserved.
+ */
+int regione_rikv_store_e4m3(const regione_bf16* k_full, const regione_bf16* v_full,
+                            const int32_t* keep_rows, const int32_t* n_keep,
+                            int B, int N_full, int Nc_cap, int H, int D,
+                            uint8_t* k_q, uint8_t* v_q, float* k_scale, float* v_scale,
+                            int32_t* dev_status, void* stream);
+int regione_rikv_load_e4m3(const uint8_t* k_q, const uint8_t* v_q, const float* k_scale,
+                           const float* v_scale, const int32_t* n_keep,
+                           int B, int Nc_cap, int H, int D,
+                           regione_bf16* k_cache, regione_bf16* v_cache,
+                           int32_t* dev_status, void* stream);
+
+/*
  * Region attention with the Region-Instruction KV cache (Sec. 4, "Region-Aware
  * Generation", the attention equation):
  *     out[b,i,h,:] = sum_j softmax_j( scale * q[b,i,h,:] . k_j ) * v_j

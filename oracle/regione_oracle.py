@@ -13,7 +13,8 @@ Pins (see tests, marker "not gpu"): straight-line identity, Euler invariance,
 planted-mask recovery, index invariants, scatter(gather) round trip, plain
 copy for the identity keep list, brute-force loops on tiny shapes, agreement
 with a library softmax-attention, split/permutation invariance, uniform-key
-mean, dominant-key selection, the row-membership counts and partition-of-the-sequence
+mean, dominant-key selection, the E4M3 code table against a library's and its round trip,
+the row-membership counts and partition-of-the-sequence
 property, the gamma = 1 closed form of the appendix, planted
 decay corrections for the gamma fit, and the zero-edit / full-edit merge cases.
 Every function has such a pin.  Two of them implement a *reading* where the paper
@@ -216,6 +217,85 @@ def rikv_store(k_full, v_full, keep_rows, n_keep):
     keep_rows [B, cap]; returns (k_cache, v_cache) [B, cap, H, D], NaN past n_keep[b].
     """
     return gather(k_full, keep_rows, n_keep), gather(v_full, keep_rows, n_keep)
+
+
+# ----------------------------------------------------------------------------
+# 8-bit (E4M3) variant of the cache.  The paper keeps the cache in the model's precision; this is
+# the storage variant of the library, stated here from the published format: 1 sign bit, 4 exponent
+# bits (bias 7), 3 mantissa bits, exponent field 0 = subnormal, largest finite value 448, no
+# infinities (sign.1111.111 is NaN).
+# ----------------------------------------------------------------------------
+
+
+def e4m3_decode(code):
+    """Value of an E4M3 code (uint8 array) in float64; the two NaN codes give NaN."""
+    c = np.asarray(code).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 15
+    m = c & 7
+    mag = np.where(e == 0, m / 8.0 * 2.0 ** -6, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7.0))
+    return np.where((e == 15) & (m == 7), np.nan, sign * mag)
+
+
+def e4m3_encode(y):
+    """Nearest E4M3 code of each value (ties to the even mantissa), magnitudes above 448 saturate
+    at 448.  A plain search over the 127 non-negative finite codes, no bit tricks."""
+    y = _f64(y)
+    grid = e4m3_decode(np.arange(127, dtype=np.uint8))          # 0 .. 448, ascending
+    a = np.minimum(np.abs(y), 448.0)
+    hi = np.searchsorted(grid, a, side="left")                   # first code with value >= a
+    hi = np.minimum(hi, 126)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = a - grid[lo], grid[hi] - a
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))   # tie: the code with an even last bit
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    return np.where(np.signbit(y), code | 0x80, code).astype(np.uint8)
+
+
+def kv_scale_exponent(amax):
+    """k of the power-of-two scale 2^k of one (row, head): the smallest k with amax / 2^k <= 448
+    (k = 0 for amax = 0, k >= -100)."""
+    amax = float(amax)
+    if not amax > 0.0:
+        return 0
+    k = -200
+    while amax / 2.0 ** k > 448.0:
+        k += 1
+    return max(k, -100)
+
+
+def rikv_store_e4m3(k_full, v_full, keep_rows, n_keep):
+    """The retained rows of K and V as E4M3 codes with one scale per (row, head).
+
+    Returns (k_codes, v_codes uint8 [B, cap, H, D], k_scale, v_scale float64 [B, cap, H]); entries past
+    n_keep[b] are 0 / NaN."""
+    outs = []
+    for full in (k_full, v_full):
+        full = _f64(full)
+        B, _, H, D = full.shape
+        cap = np.shape(keep_rows)[1]
+        codes = np.zeros((B, cap, H, D), np.uint8)
+        scale = np.full((B, cap, H), np.nan)
+        for b in range(B):
+            for j in range(int(n_keep[b])):
+                row = full[b, keep_rows[b][j]]
+                for h in range(H):
+                    s = 2.0 ** kv_scale_exponent(np.max(np.abs(row[h])))
+                    scale[b, j, h] = s
+                    codes[b, j, h] = e4m3_encode(row[h] / s)
+        outs.append((codes, scale))
+    return outs[0][0], outs[1][0], outs[0][1], outs[1][1]
+
+
+def rikv_load_e4m3(k_codes, v_codes, k_scale, v_scale, n_keep):
+    """The cache the attention sees: code value times the row-and-head scale (NaN past n_keep[b])."""
+    res = []
+    for codes, scale in ((k_codes, k_scale), (v_codes, v_scale)):
+        out = e4m3_decode(codes) * np.asarray(scale, np.float64)[..., None]
+        for b in range(out.shape[0]):
+            out[b, int(n_keep[b]):] = np.nan
+        res.append(out)
+    return res[0], res[1]
 
 
 # ----------------------------------------------------------------------------

@@ -36,6 +36,8 @@ SIGNATURES = {
     "regione_gather_multi": (c_int, [_P, _P, c_int, _P, _P, c_int, c_int64, c_int64, c_int64, c_int64, _P, _P]),
     "regione_scatter": (c_int, [_P, _P, _P, c_int, c_int64, c_int64, c_int64, c_int64, _P, _P, _P]),
     "regione_rikv_store": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
+    "regione_rikv_store_e4m3": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P, _P, _P]),
+    "regione_rikv_load_e4m3": (c_int, [_P, _P, _P, _P, _P, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
     "regione_region_attention_workspace": (c_size_t, [c_int] * 6),
     "regione_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, c_size_t, _P, _P]),
     "regione_region_attention_scatter": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, c_int, _P, _P, c_size_t, _P, _P]),
@@ -236,6 +238,31 @@ def rikv_store(k_full, v_full, keep_rows, n_keep, k_cache, v_cache, dev_status=N
         _ptr(n_keep, torch.int32), B, n_full, k_cache.shape[1], H, D, _ptr(k_cache, bf, "k_cache"),
         _ptr(v_cache, bf, "v_cache"), _ptr(dev_status, torch.int32), _stream(stream)),
         "regione_rikv_store")
+
+
+def rikv_store_e4m3(k_full, v_full, keep_rows, n_keep, k_q, v_q, k_scale, v_scale, dev_status=None, stream=None):
+    """``rikv_store`` into an 8-bit (E4M3) cache with one power-of-two scale per (row, head)."""
+    torch = _torch()
+    bf = torch.bfloat16
+    B, n_full, H, D = k_full.shape
+    _check(load().regione_rikv_store_e4m3(
+        _ptr(k_full, bf, "k_full"), _ptr(v_full, bf, "v_full"), _ptr(keep_rows, torch.int32),
+        _ptr(n_keep, torch.int32), B, n_full, k_q.shape[1], H, D, _ptr(k_q, torch.uint8, "k_q"),
+        _ptr(v_q, torch.uint8, "v_q"), _ptr(k_scale, torch.float32, "k_scale"),
+        _ptr(v_scale, torch.float32, "v_scale"), _ptr(dev_status, torch.int32), _stream(stream)),
+        "regione_rikv_store_e4m3")
+
+
+def rikv_load_e4m3(k_q, v_q, k_scale, v_scale, n_keep, k_cache, v_cache, dev_status=None, stream=None):
+    """Widens an 8-bit cache back to bf16 (exactly the quantised values) for the attention."""
+    torch = _torch()
+    bf = torch.bfloat16
+    B, cap, H, D = k_q.shape
+    _check(load().regione_rikv_load_e4m3(
+        _ptr(k_q, torch.uint8, "k_q"), _ptr(v_q, torch.uint8, "v_q"), _ptr(k_scale, torch.float32, "k_scale"),
+        _ptr(v_scale, torch.float32, "v_scale"), _ptr(n_keep, torch.int32), B, cap, H, D,
+        _ptr(k_cache, bf, "k_cache"), _ptr(v_cache, bf, "v_cache"), _ptr(dev_status, torch.int32),
+        _stream(stream)), "regione_rikv_load_e4m3")
 
 
 def region_attention_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D) -> int:

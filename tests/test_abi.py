@@ -16,7 +16,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _header_symbols():
     text = open(os.path.join(ROOT, "include", "regione.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(regione_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(regione_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
@@ -59,6 +59,21 @@ def test_argument_validation_happens_on_the_host():
     assert lib.regione_scatter(fake, fake, fake, 1, 8, 4, 8, 32, fake, null, null) == binding.INVALID_ARG
     assert lib.regione_rikv_store(fake, fake, fake, fake, 1, 8, 8, 3, 3, fake, fake, null, null) \
         == binding.UNSUPPORTED
+    # the 8-bit cache: head sizes 64 and 128 only, 16-byte aligned buffers, counts required
+    assert lib.regione_rikv_store_e4m3(fake, fake, fake, fake, 1, 8, 8, 3, 96, fake, fake, fake, fake, null,
+                                       null) == binding.UNSUPPORTED
+    assert lib.regione_rikv_store_e4m3(fake, fake, fake, null, 1, 8, 8, 3, 64, fake, fake, fake, fake, null,
+                                       null) == binding.INVALID_ARG
+    assert lib.regione_rikv_store_e4m3(fake, fake, fake, fake, 1, 8, 8, 3, 64, odd, fake, fake, fake, null,
+                                       null) == binding.INVALID_ARG
+    assert lib.regione_rikv_store_e4m3(fake, fake, fake, fake, 0, 8, 8, 3, 64, fake, fake, fake, fake, null,
+                                       null) == binding.OK                        # nothing to do
+    assert lib.regione_rikv_load_e4m3(fake, fake, fake, fake, fake, 1, 8, 3, 32, fake, fake, null, null) \
+        == binding.UNSUPPORTED
+    assert lib.regione_rikv_load_e4m3(fake, fake, null, fake, fake, 1, 8, 3, 128, fake, fake, null, null) \
+        == binding.INVALID_ARG
+    assert lib.regione_rikv_load_e4m3(fake, fake, fake, fake, fake, 1, 0, 3, 128, fake, fake, null, null) \
+        == binding.OK
     assert lib.regione_region_attention(fake, fake, fake, fake, fake, fake, fake, fake, 1, 8, 8, 8, 2, 96,
                                         0.0, fake, null, 0, null, null) == binding.UNSUPPORTED
     assert lib.regione_region_attention(fake, null, null, fake, fake, fake, fake, fake, 1, 8, 8, 8, 2, 64,
