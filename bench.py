@@ -443,45 +443,52 @@ def full_step_row(torch, binding, synth, flush_l2, to_dev, peaks, iters=10):
 
 
 def kv_e4m3_row(torch, binding, synth, flush_l2, to_dev, peaks, iters=10):
-    """The 8-bit (E4M3) variant of the cache on the headline layer's shape: the store that quantises the
-    retained rows, the pass that widens them back to bf16 before a region step's attention, both as HBM
-    passes against the measured copy bandwidth, and the bytes one cached layer holds in either form."""
-    wl = synth.WORKLOADS[2]
-    qkv = synth.make_qkv_full(wl)
-    k, v = to_dev(qkv["k"]), to_dev(qkv["v"])
-    del qkv
-    n, H, D = wl.n_full, wl.heads, wl.head_dim
+    """The 8-bit (E4M3) variant of the cache on the headline layer's shape and on the batch of four large
+    requests: the store that quantises the retained rows, the pass that widens them back to bf16 before a
+    region step's attention, both as HBM passes against the measured copy bandwidth, and the bytes one
+    cached layer holds in either form."""
     i32, bf = torch.int32, torch.bfloat16
-    kept = n - int(round(wl.ratios[0] * wl.n_img))
-    keep = torch.arange(kept, dtype=i32, device="cuda").reshape(1, kept) + (n - kept)
-    n_keep = torch.tensor([kept], dtype=i32, device="cuda")
-    kq = torch.empty((1, kept, H, D), dtype=torch.uint8, device="cuda"); vq = torch.empty_like(kq)
-    ks = torch.empty((1, kept, H), dtype=torch.float32, device="cuda"); vs = torch.empty_like(ks)
-    kc = torch.empty((1, kept, H, D), dtype=bf, device="cuda"); vc = torch.empty_like(kc)
-    st = torch.zeros(1, dtype=i32, device="cuda")
-    calls = (("rikv_store_bf16", 2 * 2 * 2 * kept * H * D,
-              lambda: binding.rikv_store(k, v, keep, n_keep, kc, vc, dev_status=st)),
-             ("rikv_store_e4m3", 2 * kept * H * (3 * D + 4),
-              lambda: binding.rikv_store_e4m3(k, v, keep, n_keep, kq, vq, ks, vs, dev_status=st)),
-             ("rikv_load_e4m3", 2 * kept * H * (3 * D + 4),
-              lambda: binding.rikv_load_e4m3(kq, vq, ks, vs, n_keep, kc, vc, dev_status=st)))
-    res = dict(workload="config 2 shape, one layer's retained rows", kept_rows=kept,
-               cache_bytes_bf16=2 * 2 * kept * H * D, cache_bytes_e4m3=2 * kept * H * (D + 4))
-    for name, nbytes, fn in calls:
-        for _ in range(3):
-            fn()
-        ts = []
-        for _ in range(iters):
-            flush_l2()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(); fn(); b.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b) * 1e3)
-        us = float(np.median(ts))
-        res[name] = dict(us=round(us, 1), algorithmic_bytes=nbytes, gbs=round(nbytes / us / 1e3, 1),
-                         frac_of_measured_hbm=round(nbytes / us / 1e3 / peaks["hbm_gbs"], 3))
-    assert int(st[0]) == 0
-    return res
+    out = dict(workload="one layer's retained rows: bf16 store, E4M3 store, E4M3 widening", sizes=[])
+    for cfg in (2, 5):
+        wl = synth.WORKLOADS[cfg]
+        qkv = synth.make_qkv_full(wl)
+        k, v = to_dev(qkv["k"]), to_dev(qkv["v"])
+        del qkv
+        B, n, H, D = wl.batch, wl.n_full, wl.heads, wl.head_dim
+        kept = n - int(round(wl.ratios[0] * wl.n_img))
+        keep = (torch.arange(kept, dtype=i32, device="cuda") + (n - kept)).repeat(B, 1).contiguous()
+        n_keep = torch.full((B,), kept, dtype=i32, device="cuda")
+        kq = torch.empty((B, kept, H, D), dtype=torch.uint8, device="cuda"); vq = torch.empty_like(kq)
+        ks = torch.empty((B, kept, H), dtype=torch.float32, device="cuda"); vs = torch.empty_like(ks)
+        kc = torch.empty((B, kept, H, D), dtype=bf, device="cuda"); vc = torch.empty_like(kc)
+        st = torch.zeros(1, dtype=i32, device="cuda")
+        rows = B * kept
+        calls = (("rikv_store_bf16", 2 * 2 * 2 * rows * H * D,
+                  lambda: binding.rikv_store(k, v, keep, n_keep, kc, vc, dev_status=st)),
+                 ("rikv_store_e4m3", 2 * rows * H * (3 * D + 4),
+                  lambda: binding.rikv_store_e4m3(k, v, keep, n_keep, kq, vq, ks, vs, dev_status=st)),
+                 ("rikv_load_e4m3", 2 * rows * H * (3 * D + 4),
+                  lambda: binding.rikv_load_e4m3(kq, vq, ks, vs, n_keep, kc, vc, dev_status=st)))
+        res = dict(config=cfg, requests=B, kept_rows=kept, cache_bytes_bf16=2 * 2 * rows * H * D,
+                   cache_bytes_e4m3=2 * rows * H * (D + 4))
+        for name, nbytes, fn in calls:
+            for _ in range(3):
+                fn()
+            ts = []
+            for _ in range(iters):
+                flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3)
+            us = float(np.median(ts))
+            res[name] = dict(us=round(us, 1), algorithmic_bytes=nbytes, gbs=round(nbytes / us / 1e3, 1),
+                             frac_of_measured_hbm=round(nbytes / us / 1e3 / peaks["hbm_gbs"], 3))
+        assert int(st[0]) == 0
+        out["sizes"].append(res)
+        del k, v, kq, vq, kc, vc
+        torch.cuda.empty_cache()
+    return out
 
 
 def loop_row(torch, binding, synth, to_dev):
