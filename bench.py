@@ -353,6 +353,18 @@ def per_config_rows(torch, binding, synth, flush_l2, to_dev, peaks, steps=12):
         st_us = float(np.mean([e[0].elapsed_time(e[3]) for e in ev]) * 1e3)
         at_us = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]) * 1e3)
         tf = fl / at_us / 1e6
+        # the same step without the cache store: Algorithm 1 writes the cache at full steps only, a run of
+        # region steps in between reuses it
+        reuse = []
+        for i in range(steps):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            step.run(x_t, v, ref, dq, dk, dv, lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0, store_cache=False)
+            b.record()
+            reuse.append((a, b))
+        torch.cuda.synchronize()
+        reuse_us = float(np.mean([a.elapsed_time(b) for a, b in reuse]) * 1e3)
         graph_us = None
         if cfg == 1:
             # the tiny layer's step is launch-bound (8 kernels of a few microseconds each): the same step
@@ -375,7 +387,8 @@ def per_config_rows(torch, binding, synth, flush_l2, to_dev, peaks, steps=12):
             assert int(step.dev_status[0]) == 0
         rows.append(dict(config=cfg, workload=wl.name, membership=membership, batch=wl.batch,
                          n_q=int(n_q[0]), n_kv=int(n_kv[0]), heads=wl.heads, head_dim=wl.head_dim,
-                         step_us=round(st_us, 1), step_us_cuda_graph=graph_us,
+                         step_us=round(st_us, 1), step_us_cache_reused=round(reuse_us, 1),
+                         step_us_cuda_graph=graph_us,
                          attention_us=round(at_us, 1), attention_tflops=round(tf, 1),
                          attention_frac_of_measured_burst=round(tf / peaks["bf16_tflops"], 3),
                          attention_frac_of_nominal_2250=round(tf / NOMINAL_BF16_TFLOPS, 3),
@@ -714,6 +727,18 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    # the headline step without its cache store (a region step between two full steps of Algorithm 1)
+    reuse = []
+    for _ in range(min(steps, 50)):
+        flush_l2()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        step.run(d["x_t"], d["v"], d["ref"], d["q"], d["k"], d["vv"], t, scale, dt, dt_u, store_cache=False)
+        b.record()
+        reuse.append((a, b))
+    torch.cuda.synchronize()
+    reuse_us = float(np.mean([a.elapsed_time(b) for a, b in reuse]) * 1e3)
+
     peaks = measured_peaks()
     hbm_kernels = None
     if world == 1 and not args.no_hbm_sweep:
@@ -757,6 +782,7 @@ def run_ours(args):
                 step_us=dict(mean=float(step_ms.mean() * 1e3), min=float(step_ms.min() * 1e3),
                              median=float(np.median(step_ms) * 1e3)),
                 attention_us=dict(mean=attn_us, min=float(attn_ms.min() * 1e3)),
+                step_us_cache_reused=reuse_us,
                 wall_s_timed_region=wall)
     print(json.dumps(line))
     if world > 1:

@@ -89,7 +89,10 @@ class RegionStep:
         self._fork, self._join = torch.cuda.Event(), torch.cuda.Event()
         self.attention_events = None      # optional (start, stop) pair recorded around the attention
 
-    def run(self, x_t, v, ref, q_full, k_full, v_full, t, scale, dt, dt_unedited, stream=None):
+    def run(self, x_t, v, ref, q_full, k_full, v_full, t, scale, dt, dt_unedited, stream=None,
+            store_cache=True):
+        """One region-aware step.  ``store_cache=False`` leaves the cache as the last storing call wrote
+        it (Algorithm 1 refreshes it at full steps only; valid while the partition is unchanged)."""
         import torch
         s = self.shp
         st = self.dev_status
@@ -112,8 +115,9 @@ class RegionStep:
                          dev_status=st, stream=side)
         b.merge(x_t, v, self.x_e, self.slot, dt_unedited, self.x_out, dev_status=st, stream=side)
         self._join.record(side)
-        b.rikv_store(k_full, v_full, self.cache_rows, self.n_cache, self.k_cache, self.v_cache,
-                     dev_status=st, stream=stream)
+        if store_cache:
+            b.rikv_store(k_full, v_full, self.cache_rows, self.n_cache, self.k_cache, self.v_cache,
+                         dev_status=st, stream=stream)
         b.gather_multi([q_full, k_full, v_full], self.query_rows, self.n_q,
                        [self.q_e, self.k_fresh, self.v_fresh], dev_status=st, stream=stream)
         if self.attention_events is not None:
@@ -125,5 +129,5 @@ class RegionStep:
         if self.attention_events is not None:
             self.attention_events[1].record(stream)
         main.wait_event(self._join)
-        self.launches += 8           # kernels launched (the attention call launches two)
+        self.launches += 8 if store_cache else 7     # kernels launched (the attention call launches two)
         return self.x_out

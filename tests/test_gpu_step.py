@@ -69,6 +69,37 @@ def test_zero_edit_mask_is_one_step_prediction_everywhere():
     run_step(synth.scaled_workload(synth.WORKLOADS[2], grid=(16, 16), n_text=16, heads=2), ratio=0.0)
 
 
+def test_step_that_reuses_the_cache_of_an_earlier_step():
+    """Algorithm 1 refreshes the cache at full steps only: a step run with ``store_cache=False`` after a
+    storing step, on new Q / K / V of a later sampler step, attends over the fresh rows of the new tensors
+    and the cached rows of the old ones (oracle: attention with the first step's cache), in 7 launches."""
+    import torch
+    from oracle import regione_oracle as orc
+    wl = synth.scaled_workload(synth.WORKLOADS[2], grid=(24, 24), n_text=70, heads=4)
+    lat = synth.make_latents(wl)
+    old, new = synth.make_qkv_full(wl), synth.make_qkv_full(wl, stream=1)
+    t, scale, dt, dt_u = lat["t"], 0.97, 1.0 / 28.0, 5.0 / 28.0
+    d = {k: dev_bf16(lat[k]) for k in ("x_t", "v", "ref")}
+    cap = plan_capacity(d["x_t"], d["v"], d["ref"], t, binding.METRIC_COSINE, wl.threshold)
+    step = RegionStep(StepShapes(wl.batch, wl.n_img, wl.n_text, wl.n_ref, wl.channels, wl.heads, wl.head_dim,
+                                 cap, binding.METRIC_COSINE, wl.threshold, binding.ROWS_EDITED_QUERIES))
+    step.run(d["x_t"], d["v"], d["ref"], *(dev_bf16(old[k]) for k in ("q", "k", "v")), t, scale, dt, dt_u)
+    before = step.launches
+    step.o_full.fill_(0)
+    step.run(d["x_t"], d["v"], d["ref"], *(dev_bf16(new[k]) for k in ("q", "k", "v")), t, scale, dt, dt_u,
+             store_cache=False)
+    torch.cuda.synchronize()
+    assert int(step.dev_status[0]) == 0 and step.launches - before == 7
+    rows = orc.region_rows(lat["mask"][0], wl.n_text, wl.n_ref, "edited_queries")
+    nq, nc = len(rows["query"]), len(rows["cache"])
+    assert int(step.n_q[0]) == nq and int(step.n_cache[0]) == nc
+    assert np.array_equal(host_f64(step.k_cache[0, :nc]), old["k"][0, rows["cache"]].astype(np.float64))
+    want = orc.region_attention(new["q"][:, rows["query"]], new["k"][:, rows["fresh"]], new["v"][:, rows["fresh"]],
+                                old["k"][:, rows["cache"]], old["v"][:, rows["cache"]], [nq], [nq], [nc])
+    got = host_f64(step.o_full[0][step.query_rows[0, :nq].long()])
+    assert_close(got, want[0, :nq], "attention over the earlier step's cache")
+
+
 def test_step_replayed_from_a_cuda_graph_matches_the_eager_step():
     """The launches of a step (each with programmatic stream serialization, two streams) captured into a
     CUDA graph and replayed give bit-identical buffers to the same step launched eagerly."""
