@@ -154,10 +154,12 @@ struct StoreParams {
 // ---- the plan every CTA (and the merge kernel) derives from the device-side counts ------------
 // Shares are cut on a cost axis measured in ticks, not in steps, so that they take about the same
 // time: a key tile of a full query pair costs kTickPair, a key tile of a pair with one live query
-// tile kTickSingle (its even and odd key tiles run side by side on the two tile roles, so it costs
-// half as much), and every item starts with kTickStart ticks that stand for the
-// drain of the previous segment and the fill of the new one (measured on the kernel).
-constexpr int kTickPair = 8, kTickSingle = 4, kTickStart = 36;
+// tile kTickSingle (its even and odd key tiles run side by side on the two tile roles; measured per
+// thread block against its share's composition: 0.55 to 0.56 of a pair's step, not half), and every
+// item starts with kTickStart ticks that stand for the drain of the previous segment and the fill of
+// the new one (measured the same way: 3.5 to 6 pair steps depending on the workload, 5 on the
+// layers of configurations 2 and 4).
+constexpr int kTickPair = 16, kTickSingle = 9, kTickStart = 80;
 
 struct ReqShape {
     int nq, nf, nc;      // clamped counts
