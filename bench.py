@@ -48,7 +48,7 @@ def measured_peaks():
 
 # DRAM bytes per attention launch on config 2 (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
 # capture of this workload), valid for the kernel source with this digest only.
-ATTENTION_TRAFFIC = dict(source_sha256_16="c8e247fbcff9abf1", config=2, dram_bytes_per_launch=205.2e6)
+ATTENTION_TRAFFIC = dict(source_sha256_16="923074f802733a8a", config=2, dram_bytes_per_launch=229.5e6)
 
 
 def recorded_traffic(cfg):
