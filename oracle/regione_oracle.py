@@ -14,6 +14,7 @@ planted-mask recovery, index invariants, scatter(gather) round trip, plain
 copy for the identity keep list, brute-force loops on tiny shapes, agreement
 with a library softmax-attention, split/permutation invariance, uniform-key
 mean, dominant-key selection, the E4M3 code table against a library's and its round trip,
+the RMS normalisation against a library's and the rotary embedding's relative-position property,
 the row-membership counts and partition-of-the-sequence
 property, the gamma = 1 closed form of the appendix, planted
 decay corrections for the gamma fit, and the zero-edit / full-edit merge cases.
@@ -296,6 +297,62 @@ def rikv_load_e4m3(k_codes, v_codes, k_scale, v_scale, n_keep):
             out[b, int(n_keep[b]):] = np.nan
         res.append(out)
     return res[0], res[1]
+
+
+# ----------------------------------------------------------------------------
+# Producer of the fresh Q / K / V rows of a region step: gather, per-head RMS normalisation of Q and
+# K, rotary position embedding at the rows' own positions in the joint sequence.  The paper does not
+# state these two operations (it treats the attention layer of the editors it accelerates as given);
+# the editors apply them to Q and K of every attention layer, and what the method adds is that a
+# recomputed token keeps its position (Sec. 4 "Region-Aware Generation": the region's tokens are
+# gathered and later put back by spatial position), so the row index of the gather is also the
+# position of the rotation.  Definitions, from their publications:
+#   RMS normalisation   y = x / sqrt(mean(x^2) + eps) * w                     (per row and head, over D)
+#   rotary embedding    (a, b) -> (a cos t - b sin t, a sin t + b cos t)      for each of the D/2 pairs,
+#     pair i = elements (2i, 2i+1) ("interleaved") or (i, i + D/2) ("half"), angle t = theta[pos, i]
+# ----------------------------------------------------------------------------
+
+ROPE_INTERLEAVED = 0
+ROPE_HALF = 1
+
+
+def rms_norm(x, weight=None, eps=1e-6):
+    """x / sqrt(mean(x^2 over the last axis) + eps), times `weight` [D] if given."""
+    x = _f64(x)
+    y = x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
+    return y if weight is None else y * _f64(weight)
+
+
+def rope(x, cos, sin, layout):
+    """Rotates the D/2 pairs of the last axis of x [..., D] by the angles whose cosines and sines are
+    cos, sin [..., D/2] (broadcast against x's leading axes)."""
+    x = _f64(x)
+    D = x.shape[-1]
+    cos, sin = _f64(cos), _f64(sin)
+    out = np.empty_like(x)
+    for i in range(D // 2):
+        ia, ib = (2 * i, 2 * i + 1) if layout == ROPE_INTERLEAVED else (i, i + D // 2)
+        a, b = x[..., ia], x[..., ib]
+        out[..., ia] = a * cos[..., i] - b * sin[..., i]
+        out[..., ib] = a * sin[..., i] + b * cos[..., i]
+    return out
+
+
+def fresh_qkv(q_full, k_full, v_full, idx, n, q_weight, k_weight, eps, cos, sin, layout):
+    """Rows idx[b, :n[b]] of Q, K, V [B, N, H, D]; Q and K normalised per head and rotated by the
+    angles of their own row position (cos, sin: [N, D/2]); V copied.  NaN past n[b]."""
+    q_full, k_full = _f64(q_full), _f64(k_full)
+    B, _, H, D = q_full.shape
+    cap = np.shape(idx)[1]
+    q = np.full((B, cap, H, D), np.nan)
+    k = np.full((B, cap, H, D), np.nan)
+    for b in range(B):
+        for j in range(int(n[b])):
+            r = int(idx[b][j])
+            for h in range(H):
+                q[b, j, h] = rope(rms_norm(q_full[b, r, h], q_weight, eps), cos[r], sin[r], layout)
+                k[b, j, h] = rope(rms_norm(k_full[b, r, h], k_weight, eps), cos[r], sin[r], layout)
+    return q, k, gather(v_full, idx, n)
 
 
 # ----------------------------------------------------------------------------
