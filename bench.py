@@ -397,6 +397,7 @@ def per_config_rows(torch, binding, synth, flush_l2, to_dev, peaks, steps=12):
         torch.cuda.empty_cache()
     rows.append(full_step_row(torch, binding, synth, flush_l2, to_dev, peaks))
     rows.append(kv_e4m3_row(torch, binding, synth, flush_l2, to_dev, peaks))
+    rows.append(fresh_qkv_row(torch, binding, synth, flush_l2, to_dev, peaks))
     rows.append(loop_row(torch, binding, synth, to_dev))
     return rows
 
@@ -500,6 +501,52 @@ def kv_e4m3_row(torch, binding, synth, flush_l2, to_dev, peaks, iters=10):
         assert int(st[0]) == 0
         out["sizes"].append(res)
         del k, v, kq, vq, kc, vc
+        torch.cuda.empty_cache()
+    return out
+
+
+def fresh_qkv_row(torch, binding, synth, flush_l2, to_dev, peaks, iters=10):
+    """The producer of fresh Q / K / V rows (gather + per-head RMS normalisation + rotary embedding in one
+    pass) beside the plain gather of the same rows: at the headline layer's region step (819 rows) and as
+    an HBM pass over every row of config 5's batch (what a full step's producer moves)."""
+    i32, bf = torch.int32, torch.bfloat16
+    out = dict(workload="fresh Q/K/V rows: plain gather of three tensors, and gather + RMS norm + rotary embedding", sizes=[])
+    for cfg, all_rows in ((2, False), (5, True)):
+        wl = synth.WORKLOADS[cfg]
+        qkv = synth.make_qkv_full(wl)
+        q, k, v = (to_dev(qkv[x]) for x in ("q", "k", "v"))
+        del qkv
+        B, n, H, D = wl.batch, wl.n_full, wl.heads, wl.head_dim
+        rows = n if all_rows else int(round(wl.ratios[0] * wl.n_img))
+        idx = (torch.arange(rows, dtype=i32, device="cuda") + (0 if all_rows else wl.n_text)).repeat(B, 1).contiguous()
+        cnt = torch.full((B,), rows, dtype=i32, device="cuda")
+        pos = torch.arange(n, dtype=torch.float64, device="cuda")[:, None]
+        inv = 10000.0 ** (-torch.arange(D // 2, dtype=torch.float64, device="cuda") * 2.0 / D)
+        cos, sin = torch.cos(pos * inv).float().contiguous(), torch.sin(pos * inv).float().contiguous()
+        w = torch.ones(D, dtype=bf, device="cuda")
+        dq, dk, dv = (torch.empty((B, rows, H, D), dtype=bf, device="cuda") for _ in range(3))
+        st = torch.zeros(1, dtype=i32, device="cuda")
+        nbytes = B * rows * (3 * 2 * H * D * 2 + 4 + 2 * (D // 2) * 4)
+        calls = (("gather_multi", lambda: binding.gather_multi([q, k, v], idx, cnt, [dq, dk, dv], dev_status=st)),
+                 ("fresh_qkv", lambda: binding.fresh_qkv(q, k, v, idx, cnt, w, w, 1e-6, cos, sin, binding.ROPE_INTERLEAVED,
+                                                         dq, dk, dv, dev_status=st)))
+        res = dict(config=cfg, requests=B, rows=rows, heads=H, head_dim=D, algorithmic_bytes=nbytes)
+        for name, fn in calls:
+            for _ in range(3):
+                fn()
+            ts = []
+            for _ in range(iters):
+                flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3)
+            us = float(np.median(ts))
+            res[name] = dict(us=round(us, 1), gbs=round(nbytes / us / 1e3, 1),
+                             frac_of_measured_hbm=round(nbytes / us / 1e3 / peaks["hbm_gbs"], 3))
+        assert int(st[0]) == 0
+        out["sizes"].append(res)
+        del q, k, v, dq, dk, dv
         torch.cuda.empty_cache()
     return out
 

@@ -67,6 +67,8 @@ enum { REGIONE_METRIC_COSINE = 0, REGIONE_METRIC_L2 = 1 };
 
 /* membership of the joint sequence rows in one region-attention call */
 enum { REGIONE_ROWS_EDITED_QUERIES = 0, REGIONE_ROWS_PAPER = 1 };
+/* which elements of a head form a rotary pair: (2i, 2i+1) or (i, i + D/2) */
+enum { REGIONE_ROPE_INTERLEAVED = 0, REGIONE_ROPE_HALF = 1 };
 
 /* Library version (major*10000 + minor*100 + patch) and status names. */
 int regione_version(void);
@@ -173,6 +175,34 @@ int regione_gather_multi(const void* const* srcs, void* const* dsts, int n_tenso
                          const int32_t* idx, const int32_t* n, int B, int64_t src_rows,
                          int64_t idx_stride, int64_t dst_rows_cap, int64_t row_bytes,
                          int32_t* dev_status, void* stream);
+
+/*
+ * Producer of a region step's fresh Q / K / V rows: the gather of the recomputed tokens' rows of Q,
+ * K and V (Algorithm 1: the same E_index for all three) fused with the two operations the editors
+ * apply to Q and K before attention, per-head RMS normalisation and rotary position embedding.  The
+ * paper does not state those two (it takes the attention layer as given); what it fixes is that a
+ * recomputed token keeps its place in the joint sequence (Sec. 4 "Region-Aware Generation": region
+ * tokens are gathered and later put back by spatial position), so idx[b, j] is both the row that is
+ * gathered and the position whose angles rotate it.
+ *     y      = x / sqrt(mean_D(x^2) + eps) * weight          per row and head, fp32
+ *     (a, b) -> (a cos t - b sin t, a sin t + b cos t)       for each of the D/2 pairs of y,
+ *               t = angle i of position idx[b, j]; pair i = elements (2i, 2i+1)
+ *               (REGIONE_ROPE_INTERLEAVED) or (i, i + D/2) (REGIONE_ROPE_HALF)
+ *     q_dst[b, j, h, :] = rotate(norm(q_src[b, idx[b, j], h, :], q_weight)),  the same for K with
+ *     k_weight;  v_dst[b, j] = v_src[b, idx[b, j]]             for j < n[b]; one rounding to bf16
+ * q_src, k_src, v_src [B, N_src, H, D] bf16; idx dev int32 [B, cap]; n dev int32 [B];
+ * q_weight, k_weight dev bf16 [D] or NULL (all ones); cos_table, sin_table dev fp32 [N_src, D/2]
+ * (cosine and sine of the angles of every position: any frequency scheme, several axes included);
+ * q_dst, k_dst, v_dst [B, cap, H, D].  D is 64 or 128; all buffers 16-byte aligned.
+ * Rows past n[b] are left untouched; an index outside [0, N_src) is skipped and REGIONE_DEV_BOUNDS
+ * recorded.  Nothing is allocated; the buffers stay the caller's.
+ */
+int regione_fresh_qkv(const regione_bf16* q_src, const regione_bf16* k_src, const regione_bf16* v_src,
+                      const int32_t* idx, const int32_t* n, int B, int N_src, int cap, int H, int D,
+                      const regione_bf16* q_weight, const regione_bf16* k_weight, float eps,
+                      const float* cos_table, const float* sin_table, int rope_layout,
+                      regione_bf16* q_dst, regione_bf16* k_dst, regione_bf16* v_dst,
+                      int32_t* dev_status, void* stream);
 
 /*
  * Token scatter, the inverse placement (Sec. 4, end of the AVDCache paragraph: the

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libregione.so")
-SOURCES = ["api.cu", "partition.cu", "rowcopy.cu", "latent.cu", "gamma.cu", "kvquant.cu", "attention_simt.cu", "attention_tc.cu"]
+SOURCES = ["api.cu", "partition.cu", "rowcopy.cu", "latent.cu", "gamma.cu", "kvquant.cu", "freshqkv.cu", "attention_simt.cu", "attention_tc.cu"]
 HEADERS = ["common.cuh", "sm100_ptx.cuh"]
 
 
