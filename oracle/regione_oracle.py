@@ -21,7 +21,11 @@ decay corrections for the gamma fit, and the zero-edit / full-edit merge cases.
 Every function has such a pin.  Two of them implement a *reading* where the paper
 leaves the operator open, and are pinned as operators only, not against the paper:
 ``open_close`` (3x3 structuring element, opening then closing) and ``gamma_fit``
-(mean of per-sample norm ratios): for those two choices, parity unpinned.
+(mean of per-sample norm ratios): for those two choices, parity unpinned.  ``rms_norm``, ``rope`` and
+``fresh_qkv`` state operations the paper does not define at all (the editors' own normalisation and
+rotary embedding of Q and K): pinned against a library routine and the rotation's textbook
+properties, parity unpinned against the paper.  The 8-bit cache functions likewise follow the
+published number format, not the paper.
 """
 from __future__ import annotations
 
