@@ -190,7 +190,11 @@ int regione_gather_multi(const void* const* srcs, void* const* dsts, int n_tenso
  *               (REGIONE_ROPE_INTERLEAVED) or (i, i + D/2) (REGIONE_ROPE_HALF)
  *     q_dst[b, j, h, :] = rotate(norm(q_src[b, idx[b, j], h, :], q_weight)),  the same for K with
  *     k_weight;  v_dst[b, j] = v_src[b, idx[b, j]]             for j < n[b]; one rounding to bf16
- * q_src, k_src, v_src [B, N_src, H, D] bf16; idx dev int32 [B, cap]; n dev int32 [B];
+ * src_compact = 0: q_src, k_src, v_src [B, N_src, H, D] bf16 hold the whole sequence and row idx[b, j]
+ * is gathered (projections computed for every row, as in a full step or a synthetic layer);
+ * src_compact = 1: they are [B, cap, H, D] and row j is read (projections computed for the recomputed
+ * rows only, as a region step does); idx[b, j] is the position in both cases.  Source and
+ * destination must not overlap.  idx dev int32 [B, cap]; n dev int32 [B];
  * q_weight, k_weight dev bf16 [D] or NULL (all ones); cos_table, sin_table dev fp32 [N_src, D/2]
  * (cosine and sine of the angles of every position: any frequency scheme, several axes included);
  * q_dst, k_dst, v_dst [B, cap, H, D].  D is 64 or 128; all buffers 16-byte aligned.
@@ -199,7 +203,7 @@ int regione_gather_multi(const void* const* srcs, void* const* dsts, int n_tenso
  */
 int regione_fresh_qkv(const regione_bf16* q_src, const regione_bf16* k_src, const regione_bf16* v_src,
                       const int32_t* idx, const int32_t* n, int B, int N_src, int cap, int H, int D,
-                      const regione_bf16* q_weight, const regione_bf16* k_weight, float eps,
+                      int src_compact, const regione_bf16* q_weight, const regione_bf16* k_weight, float eps,
                       const float* cos_table, const float* sin_table, int rope_layout,
                       regione_bf16* q_dst, regione_bf16* k_dst, regione_bf16* v_dst,
                       int32_t* dev_status, void* stream);

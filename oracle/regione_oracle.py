@@ -342,21 +342,25 @@ def rope(x, cos, sin, layout):
     return out
 
 
-def fresh_qkv(q_full, k_full, v_full, idx, n, q_weight, k_weight, eps, cos, sin, layout):
-    """Rows idx[b, :n[b]] of Q, K, V [B, N, H, D]; Q and K normalised per head and rotated by the
-    angles of their own row position (cos, sin: [N, D/2]); V copied.  NaN past n[b]."""
-    q_full, k_full = _f64(q_full), _f64(k_full)
-    B, _, H, D = q_full.shape
+def fresh_qkv(q_src, k_src, v_src, idx, n, q_weight, k_weight, eps, cos, sin, layout, src_compact=False):
+    """Row j < n[b] of the result: source row idx[b, j] of Q, K, V [B, N, H, D] (or, with src_compact,
+    source row j of [B, cap, H, D]); Q and K normalised per head and rotated by the angles of
+    position idx[b, j] (cos, sin: [positions, D/2]); V copied.  NaN past n[b]."""
+    q_src, k_src, v_src = _f64(q_src), _f64(k_src), _f64(v_src)
+    B, _, H, D = q_src.shape
     cap = np.shape(idx)[1]
     q = np.full((B, cap, H, D), np.nan)
     k = np.full((B, cap, H, D), np.nan)
+    v = np.full((B, cap, H, D), np.nan)
     for b in range(B):
         for j in range(int(n[b])):
-            r = int(idx[b][j])
+            pos = int(idx[b][j])
+            r = j if src_compact else pos
             for h in range(H):
-                q[b, j, h] = rope(rms_norm(q_full[b, r, h], q_weight, eps), cos[r], sin[r], layout)
-                k[b, j, h] = rope(rms_norm(k_full[b, r, h], k_weight, eps), cos[r], sin[r], layout)
-    return q, k, gather(v_full, idx, n)
+                q[b, j, h] = rope(rms_norm(q_src[b, r, h], q_weight, eps), cos[pos], sin[pos], layout)
+                k[b, j, h] = rope(rms_norm(k_src[b, r, h], k_weight, eps), cos[pos], sin[pos], layout)
+            v[b, j] = v_src[b, r]
+    return q, k, v
 
 
 # ----------------------------------------------------------------------------

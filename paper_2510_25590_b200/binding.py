@@ -39,7 +39,7 @@ SIGNATURES = {
     "regione_rikv_store": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
     "regione_rikv_store_e4m3": (c_int, [_P, _P, _P, _P, c_int, c_int, c_int, c_int, c_int, _P, _P, _P, _P, _P, _P]),
     "regione_rikv_load_e4m3": (c_int, [_P, _P, _P, _P, _P, c_int, c_int, c_int, c_int, _P, _P, _P, _P]),
-    "regione_fresh_qkv": (c_int, [_P] * 5 + [c_int] * 5 + [_P, _P, c_float, _P, _P, c_int, _P, _P, _P, _P, _P]),
+    "regione_fresh_qkv": (c_int, [_P] * 5 + [c_int] * 6 + [_P, _P, c_float, _P, _P, c_int, _P, _P, _P, _P, _P]),
     "regione_region_attention_workspace": (c_size_t, [c_int] * 6),
     "regione_region_attention": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, _P, c_size_t, _P, _P]),
     "regione_region_attention_scatter": (c_int, [_P] * 8 + [c_int] * 6 + [c_float, _P, c_int, _P, _P, c_size_t, _P, _P]),
@@ -268,20 +268,25 @@ def rikv_load_e4m3(k_q, v_q, k_scale, v_scale, n_keep, k_cache, v_cache, dev_sta
 
 
 def fresh_qkv(q_src, k_src, v_src, idx, n, q_weight, k_weight, eps, cos_table, sin_table, rope_layout,
-              q_dst, k_dst, v_dst, dev_status=None, stream=None):
-    """Gather of the recomputed rows of Q, K, V with the per-head RMS normalisation and the rotary
-    embedding of Q and K (angles of the rows' own positions) in the same pass."""
+              q_dst, k_dst, v_dst, src_compact=False, dev_status=None, stream=None):
+    """Rows of Q, K, V of a region step with the per-head RMS normalisation and the rotary embedding of
+    Q and K (angles of position idx[b, j]) in one pass.  ``src_compact``: the sources already hold the
+    rows in order (row j), otherwise row idx[b, j] of the whole sequence is gathered."""
     torch = _torch()
     bf, f32 = torch.bfloat16, torch.float32
-    B, n_src, H, D = q_src.shape
-    if cos_table.shape != (n_src, D // 2) or sin_table.shape != (n_src, D // 2):
-        raise RegionEError("cos_table and sin_table must be [N_src, D / 2]")
+    B, src_rows, H, D = q_src.shape
+    n_pos = cos_table.shape[0]
+    if cos_table.shape != (n_pos, D // 2) or sin_table.shape != (n_pos, D // 2):
+        raise RegionEError("cos_table and sin_table must be [positions, D / 2]")
+    if (src_compact and src_rows != idx.shape[1]) or (not src_compact and src_rows != n_pos):
+        raise RegionEError("source rows must match the index capacity (compact) or the table (gathered)")
     _check(load().regione_fresh_qkv(
         _ptr(q_src, bf, "q_src"), _ptr(k_src, bf, "k_src"), _ptr(v_src, bf, "v_src"), _ptr(idx, torch.int32),
-        _ptr(n, torch.int32), B, n_src, idx.shape[1], H, D, _ptr(q_weight, bf, "q_weight"),
-        _ptr(k_weight, bf, "k_weight"), float(eps), _ptr(cos_table, f32, "cos_table"),
-        _ptr(sin_table, f32, "sin_table"), int(rope_layout), _ptr(q_dst, bf, "q_dst"), _ptr(k_dst, bf, "k_dst"),
-        _ptr(v_dst, bf, "v_dst"), _ptr(dev_status, torch.int32), _stream(stream)), "regione_fresh_qkv")
+        _ptr(n, torch.int32), B, n_pos, idx.shape[1], H, D, 1 if src_compact else 0,
+        _ptr(q_weight, bf, "q_weight"), _ptr(k_weight, bf, "k_weight"), float(eps),
+        _ptr(cos_table, f32, "cos_table"), _ptr(sin_table, f32, "sin_table"), int(rope_layout),
+        _ptr(q_dst, bf, "q_dst"), _ptr(k_dst, bf, "k_dst"), _ptr(v_dst, bf, "v_dst"),
+        _ptr(dev_status, torch.int32), _stream(stream)), "regione_fresh_qkv")
 
 
 def region_attention_workspace(B, Nq_cap, Nf_cap, Nc_cap, H, D) -> int:

@@ -36,7 +36,7 @@ template <int D, bool HALF>
 __global__ void __launch_bounds__(kFreshThreads, 4)
 fresh_qkv_kernel(const uint16_t* __restrict__ q_src, const uint16_t* __restrict__ k_src,
                  const uint16_t* __restrict__ v_src, const int32_t* __restrict__ idx,
-                 const int32_t* __restrict__ n, int N_src, int cap, int H,
+                 const int32_t* __restrict__ n, int N_src, int cap, int H, int src_compact,
                  const uint16_t* __restrict__ q_weight, const uint16_t* __restrict__ k_weight, float eps,
                  const float* __restrict__ cos_t, const float* __restrict__ sin_t,
                  uint16_t* __restrict__ q_dst, uint16_t* __restrict__ k_dst, uint16_t* __restrict__ v_dst,
@@ -90,7 +90,9 @@ fresh_qkv_kernel(const uint16_t* __restrict__ q_src, const uint16_t* __restrict_
     if (q_weight != nullptr) wq = *reinterpret_cast<const uint4*>(q_weight + 8 * g);
     if (k_weight != nullptr) wk = *reinterpret_cast<const uint4*>(k_weight + 8 * g);
 
-    const size_t src_off = ((size_t)b * N_src + row) * H * D, dst_off = ((size_t)b * cap + j) * H * D;
+    // source rows: taken at the index (a gather from the whole sequence), or already gathered (row j)
+    const size_t dst_off = ((size_t)b * cap + j) * H * D;
+    const size_t src_off = src_compact ? dst_off : ((size_t)b * N_src + row) * H * D;
     const int per_tensor = H * kLanesPerHead, total = 2 * per_tensor;   // 16-byte pieces of Q, then of K
     // V is a plain copy; its loads are issued first and stored last, so that they are in flight while
     // the pieces of Q and K are worked on
@@ -164,8 +166,9 @@ using namespace regione;
 
 extern "C" int regione_fresh_qkv(const regione_bf16* q_src, const regione_bf16* k_src,
                                  const regione_bf16* v_src, const int32_t* idx, const int32_t* n, int B,
-                                 int N_src, int cap, int H, int D, const regione_bf16* q_weight,
-                                 const regione_bf16* k_weight, float eps, const float* cos_table,
+                                 int N_src, int cap, int H, int D, int src_compact,
+                                 const regione_bf16* q_weight, const regione_bf16* k_weight, float eps,
+                                 const float* cos_table,
                                  const float* sin_table, int rope_layout, regione_bf16* q_dst,
                                  regione_bf16* k_dst, regione_bf16* v_dst, int32_t* dev_status,
                                  void* stream) {
@@ -185,7 +188,7 @@ extern "C" int regione_fresh_qkv(const regione_bf16* q_src, const regione_bf16* 
     const bool half = rope_layout == REGIONE_ROPE_HALF;
 #define REGIONE_FRESH_LAUNCH(DD, HH)                                                                       \
     launch_overlapped(fresh_qkv_kernel<DD, HH>, grid, block, 0, st, q_src, k_src, v_src, idx, n, N_src, cap, H, \
-                      q_weight, k_weight, eps, cos_table, sin_table, q_dst, k_dst, v_dst, dev_status)
+                      src_compact, q_weight, k_weight, eps, cos_table, sin_table, q_dst, k_dst, v_dst, dev_status)
     const cudaError_t e = D == 128 ? (half ? REGIONE_FRESH_LAUNCH(128, true) : REGIONE_FRESH_LAUNCH(128, false))
                                    : (half ? REGIONE_FRESH_LAUNCH(64, true) : REGIONE_FRESH_LAUNCH(64, false));
 #undef REGIONE_FRESH_LAUNCH

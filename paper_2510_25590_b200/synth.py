@@ -311,3 +311,44 @@ def gamma_table(T: int = 28, kind: str = "ones", seed: int = 7) -> np.ndarray:
         return np.ones(T + 1, dtype=np.float64)
     rng = np.random.Generator(np.random.Philox(key=seed))
     return 0.90 + 0.10 * rng.random(T + 1)
+
+
+# ----------------------------------------------------------------------------
+# random weights of the stand-in transformer stack of the sampler-loop configuration
+# ----------------------------------------------------------------------------
+
+
+def rope_tables(n_pos: int, head_dim: int, base: float = 10000.0):
+    """cos / sin [n_pos, head_dim / 2] float32 of the angles position * base^(-2i / head_dim)."""
+    inv = base ** (-np.arange(head_dim // 2, dtype=np.float64) * 2.0 / head_dim)
+    th = np.arange(n_pos, dtype=np.float64)[:, None] * inv[None, :]
+    return np.cos(th).astype(np.float32), np.sin(th).astype(np.float32)
+
+
+def mmdit_weight_shapes(hidden: int, head_dim: int, channels: int, n_text: int, blocks: int, mlp_ratio: int = 4):
+    """Name -> (shape, standard deviation, mean) of every tensor of the stand-in stack (two weight sets
+    per block: index 0 for the text rows, 1 for the image and reference rows)."""
+    hd, m = hidden, mlp_ratio * hidden
+    sh = {"text_emb": ((n_text, hd), 1.0, 0.0), "w_in": ((channels, hd), channels ** -0.5, 0.0),
+          "b_in": ((hd,), 0.1, 0.0), "ref_emb": ((hd,), 0.5, 0.0), "t_a": ((hd,), 1.0, 0.0), "t_b": ((hd,), 1.0, 0.0),
+          "w_out": ((hd, channels), hd ** -0.5, 0.0)}
+    for l in range(blocks):
+        sh[f"qn{l}"] = ((head_dim,), 0.1, 1.0)
+        sh[f"kn{l}"] = ((head_dim,), 0.1, 1.0)
+        for s in range(2):
+            sh[f"mod{l}_{s}"] = ((hd, 6 * hd), 0.5 * hd ** -0.5, 0.0)
+            sh[f"qkv{l}_{s}"] = ((hd, 3 * hd), hd ** -0.5, 0.0)
+            sh[f"o{l}_{s}"] = ((hd, hd), hd ** -0.5, 0.0)
+            sh[f"fc1_{l}_{s}"] = ((hd, m), hd ** -0.5, 0.0)
+            sh[f"fc2_{l}_{s}"] = ((m, hd), m ** -0.5, 0.0)
+    return sh
+
+
+def make_mmdit_weights(hidden: int, head_dim: int, channels: int, n_text: int, blocks: int, mlp_ratio: int = 4,
+                       seed: int = 0):
+    """Seeded bf16-representable float32 weights of the stand-in stack (host arrays: test sizes)."""
+    rng = np.random.default_rng(seed)
+    out = {}
+    for name, (shape, std, mean) in mmdit_weight_shapes(hidden, head_dim, channels, n_text, blocks, mlp_ratio).items():
+        out[name] = bf16_round((mean + std * rng.standard_normal(shape, dtype=np.float32)).astype(np.float32))
+    return out

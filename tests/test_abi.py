@@ -60,15 +60,15 @@ def test_argument_validation_happens_on_the_host():
     assert lib.regione_rikv_store(fake, fake, fake, fake, 1, 8, 8, 3, 3, fake, fake, null, null) \
         == binding.UNSUPPORTED
     # the producer of fresh Q / K / V rows: head sizes 64 and 128, a known pair layout, tables required
-    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 96, null, null, 1e-6, fake, fake, 0,
+    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 96, 0, null, null, 1e-6, fake, fake, 0,
                                  fake, fake, fake, null, null) == binding.UNSUPPORTED
-    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 64, null, null, 1e-6, fake, fake, 2,
+    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 64, 0, null, null, 1e-6, fake, fake, 2,
                                  fake, fake, fake, null, null) == binding.INVALID_ARG
-    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 64, null, null, 1e-6, null, fake, 0,
+    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 64, 0, null, null, 1e-6, null, fake, 0,
                                  fake, fake, fake, null, null) == binding.INVALID_ARG
-    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 64, odd, null, 1e-6, fake, fake, 0,
+    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 4, 2, 64, 1, odd, null, 1e-6, fake, fake, 0,
                                  fake, fake, fake, null, null) == binding.INVALID_ARG
-    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 0, 2, 64, null, null, 1e-6, fake, fake, 1,
+    assert lib.regione_fresh_qkv(fake, fake, fake, fake, fake, 1, 8, 0, 2, 64, 1, null, null, 1e-6, fake, fake, 1,
                                  fake, fake, fake, null, null) == binding.OK          # nothing to do
     # the 8-bit cache: head sizes 64 and 128 only, 16-byte aligned buffers, counts required
     assert lib.regione_rikv_store_e4m3(fake, fake, fake, fake, 1, 8, 8, 3, 96, fake, fake, fake, fake, null,

@@ -19,15 +19,16 @@ def _tables(n_pos, D, seed):
     return np.cos(th).astype(np.float32), np.sin(th).astype(np.float32)
 
 
-def _run(q, k, v, idx, n, wq, wk, eps, cos, sin, layout):
+def _run(q, k, v, idx, n, wq, wk, eps, cos, sin, layout, src_compact=False):
     import torch
-    B, N, H, D = q.shape
+    B, _, H, D = q.shape
     cap = idx.shape[1]
     outs = [torch.full((B, cap, H, D), -3.0, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     binding.fresh_qkv(dev_bf16(q), dev_bf16(k), dev_bf16(v), dev_i32(idx), dev_i32(n),
                       None if wq is None else dev_bf16(wq), None if wk is None else dev_bf16(wk), eps,
-                      torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda(), layout, *outs, dev_status=st)
+                      torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda(), layout, *outs,
+                      src_compact=src_compact, dev_status=st)
     torch.cuda.synchronize()
     return outs, int(st[0])
 
@@ -60,6 +61,28 @@ def test_fresh_rows_match_the_oracle(D, H, weights, layout):
         assert np.array_equal(host_f64(gv)[b, :m], wantv[b, :m])                      # V: a copy, bit-exact
         assert np.all(host_f64(gv)[b, m:] == -3.0)
     assert np.all(host_f64(gk)[0, 0, 0] == 0.0)
+
+
+@pytest.mark.parametrize("layout", [binding.ROPE_INTERLEAVED, binding.ROPE_HALF])
+def test_rows_that_are_already_gathered_take_their_position_from_the_index(layout):
+    """A region step projects Q, K, V for the recomputed rows only: the sources hold row j at j, the index
+    list names the position whose angles rotate it.  Same result as gathering from the whole sequence."""
+    rng = np.random.default_rng(11 + layout)
+    B, N, cap, H, D = 2, 200, 60, 3, 128
+    q, k, v = (synth.bf16_round(rng.standard_normal((B, N, H, D), dtype=np.float32)) for _ in range(3))
+    idx = np.stack([np.sort(rng.permutation(N)[:cap]) for _ in range(B)]).astype(np.int32)
+    n = np.array([cap, 41], np.int32)
+    cos, sin = _tables(N, D, 4)
+    take = lambda a: np.stack([a[b, idx[b]] for b in range(B)])
+    (cq, ck, cv), st1 = _run(take(q), take(k), take(v), idx, n, None, None, 1e-6, cos, sin, layout, src_compact=True)
+    (gq, gk, gv), st2 = _run(q, k, v, idx, n, None, None, 1e-6, cos, sin, layout)
+    assert st1 == 0 and st2 == 0
+    import torch
+    for a, b_ in ((cq, gq), (ck, gk), (cv, gv)):
+        assert torch.equal(a.view(torch.int16), b_.view(torch.int16))           # bit-identical to the gathering form
+    want = orc.fresh_qkv(take(q), take(k), take(v), idx, n, None, None, np.float32(1e-6), cos, sin, layout, src_compact=True)
+    for b in range(B):
+        assert_close(host_f64(cq)[b, :n[b]], want[0][b, :n[b]], "compact source")
 
 
 def test_attention_over_produced_rows_matches_the_oracle_chain():

@@ -132,3 +132,15 @@ def test_fresh_rows_take_the_angles_of_their_own_position(layout):
         assert np.all(np.isnan(gq[b, n[b]:])) and np.all(np.isnan(gk[b, n[b]:])) and np.all(np.isnan(gv[b, n[b]:]))
     # position 0 has angle 0: a gathered row 0 is only normalised
     assert np.allclose(gq[0, 3], orc.rms_norm(q[0, 0], wq, 1e-6), rtol=1e-14)
+
+
+def test_compact_sources_are_the_gather_done_beforehand():
+    rng = np.random.default_rng(6)
+    B, N, H, D = 1, 9, 2, 8
+    q, k, v = (rng.standard_normal((B, N, H, D)) for _ in range(3))
+    idx = np.array([[7, 1, 4]]); n = [3]
+    th = _angles(N, D); c, s = np.cos(th), np.sin(th)
+    a = orc.fresh_qkv(q, k, v, idx, n, None, None, 1e-6, c, s, orc.ROPE_HALF)
+    b = orc.fresh_qkv(q[:, idx[0]], k[:, idx[0]], v[:, idx[0]], idx, n, None, None, 1e-6, c, s, orc.ROPE_HALF, src_compact=True)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
