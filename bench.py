@@ -399,6 +399,7 @@ def per_config_rows(torch, binding, synth, flush_l2, to_dev, peaks, steps=12):
     rows.append(kv_e4m3_row(torch, binding, synth, flush_l2, to_dev, peaks))
     rows.append(fresh_qkv_row(torch, binding, synth, flush_l2, to_dev, peaks))
     rows.append(loop_row(torch, binding, synth, to_dev))
+    rows.append(stack_loop_row(torch, binding, synth, to_dev))
     return rows
 
 
@@ -636,6 +637,55 @@ def loop_row(torch, binding, synth, to_dev):
                 loop_us_eager_python=round(float(np.median(eager)), 1),
                 loop_us_cuda_graph=round(float(np.median(graphed)), 1),
                 us_per_launch_cuda_graph=round(float(np.median(graphed)) / max(trace.launches, 1), 2))
+
+
+def stack_loop_row(torch, binding, synth, to_dev, blocks=8):
+    """Config 4 as BASELINE describes it: the 28-step loop around a stand-in stack of 8 random blocks
+    (hidden 3072, 24 heads x 128, MLP ratio 4; 256 text + 4096 image + 4096 reference tokens), once with
+    every step a full step and once under the region-aware schedule (partition after step 6 with the L2
+    threshold, cache refreshed every 5 steps, alternate region steps reused).  The blocks' GEMMs,
+    normalisations and activations are scaffold (torch); the Q / K / V producer, every attention, every
+    cache store and all latent updates are library calls.  Device time by CUDA events around the loop."""
+    from paper_2510_25590_b200 import loop as gloop
+    from paper_2510_25590_b200.mmdit_scaffold import MMDiTScaffold
+    wl = synth.WORKLOADS[4]
+    hidden, H, D, C = wl.heads * wl.head_dim, wl.heads, wl.head_dim, wl.channels
+    lat = synth.make_latents(wl, stream=4)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(4)
+    w = {}
+    for name, (shape, std, mean) in synth.mmdit_weight_shapes(hidden, D, C, wl.n_text, blocks).items():
+        w[name] = (mean + std * torch.randn(shape, device="cuda", generator=gen)).to(torch.bfloat16)
+    cos, sin = (torch.from_numpy(a).cuda() for a in synth.rope_tables(wl.n_full, D))
+    ref = to_dev(lat["ref"])
+    planted = torch.from_numpy(lat["mask"].astype(bool)).cuda()
+    model = MMDiTScaffold(w, wl.n_text, wl.n_img, wl.n_ref, H, D, blocks, cos, sin, ref, planted, binding.ROWS_PAPER)
+    noise = (torch.randn(ref.shape, device="cuda", generator=gen)).to(torch.bfloat16)
+    kinds, after = gloop.alternating_schedule()
+    T = len(kinds)
+    ts = [1.0 - k / T for k in range(T + 1)]
+    res = dict(workload="config 4: 28-step loop around 8 stand-in blocks (scaffold GEMMs by torch, path by the library)",
+               blocks=blocks, hidden=hidden, rows=wl.n_full, schedule=kinds)
+    for label, k_, after_ in (("all_full", "F" * T, T + 1), ("region_aware", kinds, after)):
+        cfg = gloop.LoopConfig(k_, after_, ts, [1.0] * (T + 1), 0.05, binding.METRIC_L2, wl.threshold)
+        lp = gloop.RegionELoop(1, wl.n_img, C, cfg)
+        model.bind(lp)
+        times = []
+        for it in range(2):                                  # the first pass warms up (GEMM plans, kernel set-up)
+            x = noise.clone()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); _, trace = lp.run(x, ref, model); b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        assert int(lp.dev_status[0]) == 0 and int(model.dev_status[0]) == 0
+        res[label] = dict(loop_ms=round(times[-1], 1), model_full_calls=trace.model_full_calls,
+                          model_region_calls=trace.model_region_calls)
+        if label == "region_aware":
+            res[label]["edited_tokens"] = int(lp.n_edit[0])
+            res[label]["mask_recovered"] = bool(torch.equal(lp.mask.bool(), planted))
+    res["speedup_region_aware_over_all_full"] = round(res["all_full"]["loop_ms"] / res["region_aware"]["loop_ms"], 2)
+    del model, w
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_ours(args):
