@@ -12,6 +12,11 @@
 // words: warp scan -> CTA scan -> cluster scan through distributed shared
 // memory, so no global scratch, no atomics and no spinning are needed and the
 // index lists come out ascending and deterministic.
+//
+// A few very long requests (at least 32768 tokens each, fewer cluster blocks than SMs) would leave
+// most of the GPU idle in that mapping.  For them the decisions are taken by a launch of their own
+// (partition_score_kernel, grid over the tokens, writes the mask bytes) and the same compaction
+// kernel follows in a form that reads the mask bytes back instead of scoring (FROM_MASK).
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -23,6 +28,8 @@ namespace regione {
 constexpr int kPartMaxThreads = 512;         // block size grows with the tokens per CTA
 constexpr int kPartMaxWords = 4096;          // 131072 tokens per CTA
 constexpr int kPartMaxCluster = 8;
+constexpr int kPartTwoLaunchTokens = 32768;  // requests at least this long may take the two-launch form
+constexpr int kPartBlocksPerGpu = 148;       // ... when their clusters are fewer blocks than a B200 has SMs
 
 // Exclusive prefix sum of popcounts of `bits[0..nwords)` into `prefix`; returns the total.
 // Every thread of the CTA must call it.  `warp_tot` is shared scratch of 33 ints.
@@ -85,7 +92,7 @@ __device__ void emit_indices(const uint32_t* bits, const int* prefix, int start,
         const int i = tl & 31;
         const int er = prefix[tl >> 5] + __popc(word & ((1u << i) - 1u));
         const bool edited = (word >> i) & 1u;
-        mask[n] = edited ? 1 : 0;
+        if (mask != nullptr) mask[n] = edited ? 1 : 0;
         if (edited) {
             slot[n] = edit_base + er;
             edit_idx[edit_base + er] = n;
@@ -123,7 +130,98 @@ __device__ __forceinline__ void accumulate_chunk(uint4 xv, uint4 vv, uint4 rv, f
     }
 }
 
+// Decisions of the 32 tokens n0 .. n0+31 of one request as a mask word (bit i = token n0 + i is
+// edited).  Called by whole warps.  L lanes share a token.
 template <int L>
+__device__ __forceinline__ uint32_t score_word(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ v,
+                                               const uint16_t* __restrict__ ref, size_t req, int n0, int N, int C,
+                                               float t, int metric, float threshold, float* __restrict__ score) {
+    const int lane = threadIdx.x & 31;
+    constexpr int TPI = 32 / L;                 // tokens per sub-iteration
+    const int sub = lane % L;                   // chunk lane inside the token group
+    const int chunks = C >> 3;                  // 16-byte chunks per token row
+    uint32_t mybit = 0;
+    // The loads of up to 4 groups of tokens are issued before any of them is reduced, so a
+    // warp keeps several kilobytes in flight (one 16-byte chunk per lane and tensor and group).
+    constexpr int G = L < 4 ? L : 4;
+#pragma unroll
+    for (int s0 = 0; s0 < L; s0 += G) {
+        uint4 xv[G], vv[G], rv[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const int tok = n0 + (s0 + g) * TPI + lane / L;
+            xv[g] = vv[g] = rv[g] = make_uint4(0, 0, 0, 0);
+            if (tok < N && sub < chunks) {
+                const size_t at = (req + tok) * (size_t)C + (sub << 3);
+                xv[g] = ld_stream128(x_t + at);
+                vv[g] = ld_stream128(v + at);
+                rv[g] = ld_stream128(ref + at);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const int s = s0 + g;
+            const int tok = n0 + s * TPI + lane / L;
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f;  // cosine: dot, |x0|^2, |ref|^2 ; l2: a0 only
+            accumulate_chunk(xv[g], vv[g], rv[g], t, metric, a0, a1, a2);
+            if (L == 32 && tok < N) {            // rows wider than 256 channels: further chunks
+                const size_t row = (req + tok) * (size_t)C;
+                for (int ch = sub + 32; ch < chunks; ch += 32)
+                    accumulate_chunk(ld_stream128(x_t + row + (ch << 3)),
+                                     ld_stream128(v + row + (ch << 3)),
+                                     ld_stream128(ref + row + (ch << 3)), t, metric, a0, a1, a2);
+            }
+#pragma unroll
+            for (int d = 1; d < L; d <<= 1) {
+                a0 += __shfl_xor_sync(0xffffffffu, a0, d);
+                a1 += __shfl_xor_sync(0xffffffffu, a1, d);
+                a2 += __shfl_xor_sync(0xffffffffu, a2, d);
+            }
+            float sc;
+            bool edited;
+            if (metric == REGIONE_METRIC_COSINE) {
+                sc = a0 / fmaxf(sqrtf(a1) * sqrtf(a2), 1e-12f);
+                edited = sc <= threshold;
+            } else {
+                sc = sqrtf(a0);
+                edited = sc > threshold;
+            }
+            const bool leader = (sub == 0) && (tok < N);
+            if (leader && score != nullptr) score[req + tok] = sc;
+            const uint32_t ballot = __ballot_sync(0xffffffffu, leader && edited);
+            if (lane / TPI == s) mybit = (ballot >> ((lane % TPI) * L)) & 1u;
+        }
+    }
+    return __ballot_sync(0xffffffffu, mybit != 0);
+}
+
+// Large requests, first of two launches: the decisions alone, over a grid that does not depend on the
+// request boundaries (blockIdx.y = request, the blocks of a request stride over its mask words).  The
+// mask bytes it writes are what the compaction launch behind it reads.
+template <int L>
+__global__ void __launch_bounds__(256)
+partition_score_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ v,
+                       const uint16_t* __restrict__ ref, int N, int C, const PerRequestF tv, int b0, int metric,
+                       float threshold, uint8_t* __restrict__ mask, float* __restrict__ score) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int b = b0 + blockIdx.y;
+    const float t = tv.v[blockIdx.y];
+    if (t != t) return;                          // NaN: this request sits the call out
+    const size_t req = (size_t)b * N;
+    const int lane = threadIdx.x & 31;
+    const int nwords = (N + 31) >> 5;
+    const int warps = (blockDim.x >> 5) * gridDim.x;
+    for (int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); w < nwords; w += warps) {
+        const uint32_t word = score_word<L>(x_t, v, ref, req, w << 5, N, C, t, metric, threshold, score);
+        const int tok = (w << 5) + lane;
+        if (tok < N) mask[req + tok] = (word >> lane) & 1u;
+    }
+}
+
+// FROM_MASK: the decisions were taken by partition_score_kernel; this launch reads the mask bytes back
+// (x_t, v, ref are not touched) and does the ordered compaction only.
+template <int L, bool FROM_MASK>
 __global__ void __launch_bounds__(kPartMaxThreads)
 partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ v,
                  const uint16_t* __restrict__ ref, int N, int C, int share, const PerRequestF tv,
@@ -148,69 +246,33 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
     if (t != t) return;                          // NaN: this request sits the call out (whole cluster)
     const int start = rank * share;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int TPI = 32 / L;                 // tokens per sub-iteration
-    const int sub = lane % L;                   // chunk lane inside the token group
-    const int chunks = C >> 3;                  // 16-byte chunks per token row
     const size_t req = (size_t)b * N;
 
     // ---- phase 1: score + decision, one mask word per 32 tokens -------------------------
-    const int nwarps = blockDim.x >> 5;
-    for (int w = warp; w < nwords; w += nwarps) {
-        const int n0 = start + (w << 5);
-        uint32_t mybit = 0;
-        // The loads of up to 4 groups of tokens are issued before any of them is reduced, so a
-        // warp keeps several kilobytes in flight (one 16-byte chunk per lane and tensor and group).
-        constexpr int G = L < 4 ? L : 4;
+    if constexpr (FROM_MASK) {
+        // a thread packs the 32 mask bytes of one word: two 16-byte loads where the word is whole and
+        // aligned, byte loads at a ragged end or an odd request offset
+        for (int w = threadIdx.x; w < nwords; w += blockDim.x) {
+            const int n0 = start + (w << 5);
+            const uint8_t* src = mask + req + n0;
+            uint32_t word = 0;
+            if (n0 + 32 <= N && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+                const uint4 lo = *reinterpret_cast<const uint4*>(src), hi = *reinterpret_cast<const uint4*>(src + 16);
+                const uint32_t x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
 #pragma unroll
-        for (int s0 = 0; s0 < L; s0 += G) {
-            uint4 xv[G], vv[G], rv[G];
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const int tok = n0 + (s0 + g) * TPI + lane / L;
-                xv[g] = vv[g] = rv[g] = make_uint4(0, 0, 0, 0);
-                if (tok < N && sub < chunks) {
-                    const size_t at = (req + tok) * (size_t)C + (sub << 3);
-                    xv[g] = ld_stream128(x_t + at);
-                    vv[g] = ld_stream128(v + at);
-                    rv[g] = ld_stream128(ref + at);
-                }
+                for (int i = 0; i < 8; ++i)      // bytes of 0 / 1 -> 4 bits: each byte's bit lands on 21 .. 24
+                    word |= (((x[i] & 0x01010101u) * 0x00204081u >> 21) & 0xFu) << (4 * i);
+            } else {
+                for (int i = 0; i < 32 && n0 + i < N; ++i) word |= (src[i] != 0 ? 1u : 0u) << i;
             }
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const int s = s0 + g;
-                const int tok = n0 + s * TPI + lane / L;
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f;  // cosine: dot, |x0|^2, |ref|^2 ; l2: a0 only
-                accumulate_chunk(xv[g], vv[g], rv[g], t, metric, a0, a1, a2);
-                if (L == 32 && tok < N) {            // rows wider than 256 channels: further chunks
-                    const size_t row = (req + tok) * (size_t)C;
-                    for (int ch = sub + 32; ch < chunks; ch += 32)
-                        accumulate_chunk(ld_stream128(x_t + row + (ch << 3)),
-                                         ld_stream128(v + row + (ch << 3)),
-                                         ld_stream128(ref + row + (ch << 3)), t, metric, a0, a1, a2);
-                }
-#pragma unroll
-                for (int d = 1; d < L; d <<= 1) {
-                    a0 += __shfl_xor_sync(0xffffffffu, a0, d);
-                    a1 += __shfl_xor_sync(0xffffffffu, a1, d);
-                    a2 += __shfl_xor_sync(0xffffffffu, a2, d);
-                }
-                float sc;
-                bool edited;
-                if (metric == REGIONE_METRIC_COSINE) {
-                    sc = a0 / fmaxf(sqrtf(a1) * sqrtf(a2), 1e-12f);
-                    edited = sc <= threshold;
-                } else {
-                    sc = sqrtf(a0);
-                    edited = sc > threshold;
-                }
-                const bool leader = (sub == 0) && (tok < N);
-                if (leader && score != nullptr) score[req + tok] = sc;
-                const uint32_t ballot = __ballot_sync(0xffffffffu, leader && edited);
-                if (lane / TPI == s) mybit = (ballot >> ((lane % TPI) * L)) & 1u;
-            }
+            bits[w] = word;
         }
-        const uint32_t word = __ballot_sync(0xffffffffu, mybit != 0);
-        if (lane == 0) bits[w] = word;
+    } else {
+        const int nwarps = blockDim.x >> 5;
+        for (int w = warp; w < nwords; w += nwarps) {
+            const uint32_t word = score_word<L>(x_t, v, ref, req, start + (w << 5), N, C, t, metric, threshold, score);
+            if (lane == 0) bits[w] = word;
+        }
     }
     __syncthreads();
 
@@ -229,7 +291,7 @@ partition_kernel(const uint16_t* __restrict__ x_t, const uint16_t* __restrict__ 
     int32_t* const q_rows = lists ? rl.query_rows + (size_t)b * rl.q_cap : nullptr;
     int32_t* const c_rows = lists ? rl.cache_rows + (size_t)b * rl.c_cap : nullptr;
     if (start < N) {
-        emit_indices(bits, prefix, start, share, N, edit_base, keep_base, mask + req,
+        emit_indices(bits, prefix, start, share, N, edit_base, keep_base, FROM_MASK ? nullptr : mask + req,
                      edit_idx + req, keep_idx + req, slot + req, rl, q_rows, c_rows, q_text, c_text);
     }
     if (rank == csize - 1 && threadIdx.x == 0) n_edit[b] = edit_base + total;
@@ -362,7 +424,7 @@ __global__ void region_rows_kernel(const int32_t* __restrict__ edit_idx,
 
 using namespace regione;
 
-template <int L>
+template <int L, bool FROM_MASK = false>
 static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st,
                                     const uint16_t* x_t, const uint16_t* v, const uint16_t* ref,
                                     int N, int C, const PerRequestF& tv, int b0, int metric,
@@ -388,7 +450,7 @@ static cudaError_t launch_partition(int csize, int B, int share, cudaStream_t st
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, partition_kernel<L>, x_t, v, ref, N, C, share, tv, b0, metric,
+    return cudaLaunchKernelEx(&cfg, partition_kernel<L, FROM_MASK>, x_t, v, ref, N, C, share, tv, b0, metric,
                               thr, mask, edit_idx, keep_idx, slot, n_edit, score, rl, dev_status);
 }
 
@@ -417,11 +479,31 @@ static int partition_impl(const regione_bf16* x_t, const regione_bf16* v, const 
         const int nb = B - b0 < kReqChunk ? B - b0 : kReqChunk;
         PerRequestF tv;
         for (int i = 0; i < nb; ++i) tv.v[i] = t[b0 + i];
+        // Few long requests: a cluster is at most 8 blocks per request, so fewer than one block per SM
+        // would read the latents (measured, 220 MB of latents: 16 requests of 131072 tokens 73 us, 2 of
+        // 1048576 369 us, against 48 us for 32 of 65536).  Then the decisions go to a launch of their own
+        // whose grid follows the tokens, and the compaction launch behind it reads the mask bytes back
+        // (56 us and 122 us on the same instances; with a block per SM or more the single launch is as
+        // fast or faster and stays).
+        const bool two_launches = N >= kPartTwoLaunchTokens && (long long)nb * csize <= kPartBlocksPerGpu;
 #define REGIONE_PART_CASE(LL)                                                                   \
     case LL:                                                                                    \
-        e = launch_partition<LL>(csize, nb, share, st, x_t, v, ref, N, C, tv, b0, metric,       \
-                                 threshold, mask, edit_idx, keep_idx, slot, n_edit, score, rl,  \
-                                 dev_status);                                                   \
+        if (two_launches) {                                                                     \
+            const int warps_per_block = 8, words_per_warp = 4;                                  \
+            const int nwords = (N + 31) / 32;                                                   \
+            const dim3 sgrid((nwords + warps_per_block * words_per_warp - 1) /                  \
+                             (warps_per_block * words_per_warp), nb);                           \
+            e = launch_overlapped(partition_score_kernel<LL>, sgrid, dim3(256), 0, st, x_t, v,  \
+                                  ref, N, C, tv, b0, metric, threshold, mask, score);           \
+            if (e == cudaSuccess)                                                               \
+                e = launch_partition<1, true>(csize, nb, share, st, x_t, v, ref, N, C, tv, b0,  \
+                                              metric, threshold, mask, edit_idx, keep_idx,      \
+                                              slot, n_edit, nullptr, rl, dev_status);           \
+        } else {                                                                                \
+            e = launch_partition<LL>(csize, nb, share, st, x_t, v, ref, N, C, tv, b0, metric,   \
+                                     threshold, mask, edit_idx, keep_idx, slot, n_edit, score,  \
+                                     rl, dev_status);                                           \
+        }                                                                                       \
         break;
         switch (L) {
             REGIONE_PART_CASE(1)
@@ -430,9 +512,7 @@ static int partition_impl(const regione_bf16* x_t, const regione_bf16* v, const 
             REGIONE_PART_CASE(8)
             REGIONE_PART_CASE(16)
             default:
-                e = launch_partition<32>(csize, nb, share, st, x_t, v, ref, N, C, tv, b0, metric,
-                                         threshold, mask, edit_idx, keep_idx, slot, n_edit, score, rl,
-                                         dev_status);
+            REGIONE_PART_CASE(32)
         }
     }
 #undef REGIONE_PART_CASE

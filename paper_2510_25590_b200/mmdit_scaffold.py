@@ -94,7 +94,7 @@ class MMDiTScaffold:
                 if n_text_rows:
                     torch.matmul(a[:n_text_rows], wq(0)[:, j * hd:(j + 1) * hd], out=out[:n_text_rows])
                 torch.matmul(a[n_text_rows:], wq(1)[:, j * hd:(j + 1) * hd], out=out[n_text_rows:])
-            k_d, v_d = (self.k_full[l], self.v_full[l]) if keep_kv else (self._k_tmp(rows), self._v_tmp(rows))
+            k_d, v_d = (self.k_full[l], self.v_full[l]) if keep_kv else (self._tmp("_ktmp", rows), self._tmp("_vtmp", rows))
             binding.fresh_qkv(q_s, k_s, v_s, positions, n_rows_dev,
                               self.w[f"qn{l}"], self.w[f"kn{l}"], 1e-6, self.cos, self.sin, binding.ROPE_INTERLEAVED,
                               q_d, k_d, v_d, src_compact=True, dev_status=self.dev_status)
@@ -106,12 +106,6 @@ class MMDiTScaffold:
             u = torch.nn.functional.gelu(self._mm(m, f"fc1_{l}", n_text_rows), approximate="tanh")
             h = (h.float() + g2 * self._mm(u, f"fc2_{l}", n_text_rows).float()).to(bf)
         return h
-
-    def _k_tmp(self, rows):
-        return self._tmp("_ktmp", rows)
-
-    def _v_tmp(self, rows):
-        return self._tmp("_vtmp", rows)
 
     def _tmp(self, name, rows):
         import torch
@@ -131,7 +125,7 @@ class MMDiTScaffold:
         import torch
         if isinstance(t, (list, tuple)):
             t, store = t[0], store[0]
-        w, n = self.w, self.n_full
+        w = self.w
         emb = lambda z: z[0] @ w["w_in"] + w["b_in"]
         h = torch.cat([w["text_emb"], emb(x), emb(self.ref) + w["ref_emb"]])
 
@@ -187,7 +181,6 @@ class MMDiTScaffold:
 
     def _blocks_compact(self, h, t, positions, n_text_rows, attend):
         """The same blocks over a compact set of rows (own buffers of that size)."""
-        import torch
         rows = h.shape[0]
         saved = self.scratch
         self.scratch = [self._tmp(f"_c{i}", rows) for i in range(5)]

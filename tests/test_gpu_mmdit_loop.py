@@ -4,7 +4,7 @@ oracle's on the same inputs, and the whole 28-step loop against the oracle loop.
 import numpy as np
 import pytest
 
-from gpu_util import assert_close, dev_bf16, dev_i32, host_f64
+from gpu_util import assert_close, dev_bf16, host_f64
 from oracle import loop_oracle, mmdit_oracle, regione_oracle as orc
 from paper_2510_25590_b200 import binding, loop as gloop, synth
 from paper_2510_25590_b200.mmdit_scaffold import MMDiTScaffold

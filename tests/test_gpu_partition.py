@@ -84,7 +84,9 @@ def test_threshold_sweep_through_the_score_distribution(metric):
 
 @pytest.mark.parametrize("N,C,B", [(1, 16, 1), (31, 16, 2), (127, 8, 1), (129, 16, 3), (513, 32, 2),
                                    (4097, 16, 1), (1000, 64, 2), (777, 256, 1), (300, 512, 2),
-                                   (150, 1024, 1), (140001, 16, 1), (9216, 16, 4)])
+                                   (150, 1024, 1), (140001, 16, 1), (9216, 16, 4),
+                                   # requests long enough for the two-launch form (decisions, then compaction)
+                                   (32768, 16, 2), (40000, 32, 3), (65539, 24, 2), (33000, 256, 1)])
 def test_ragged_sizes_and_channel_counts(N, C, B):
     rng = np.random.default_rng(N * 7 + C)
     r = rng.standard_normal((B, N, C))
@@ -171,7 +173,8 @@ def test_region_rows_match_the_oracle_membership_rule(membership):
 
 
 @pytest.mark.parametrize("membership", ["edited_queries", "paper"])
-@pytest.mark.parametrize("grid,n_text,batch", [((48, 48), 77, 3), ((64, 64), 512, 1), ((9, 7), 0, 2), ((96, 96), 33, 2)])
+@pytest.mark.parametrize("grid,n_text,batch", [((48, 48), 77, 3), ((64, 64), 512, 1), ((9, 7), 0, 2), ((96, 96), 33, 2),
+                                               ((200, 190), 40, 2)])          # 38000 tokens: the two-launch form
 def test_partition_with_row_lists_in_one_launch(membership, grid, n_text, batch):
     """regione_partition_rows = regione_partition + regione_region_rows: every output bit-exact
     against the oracle partition and the oracle row lists, tails untouched."""
@@ -247,3 +250,19 @@ def test_requests_at_their_own_sampler_times(B):
     # (otherwise this test would not notice a kernel that ignores the per-request values)
     same = run_partition(x_t, v, ref, ts[0], orc.COSINE, wl.threshold)
     assert not np.array_equal(same["score"], got["score"])
+
+
+def test_long_requests_sit_a_call_out_too():
+    """The two-launch form of long requests honours the NaN convention in both of its launches."""
+    import torch
+    rng = np.random.default_rng(12)
+    B, N, C = 3, 33000, 16
+    x_t, v, ref = (synth.bf16_round(rng.standard_normal((B, N, C)).astype(np.float32)) for _ in range(3))
+    ts = [0.6, float("nan"), 0.7]
+    got = run_partition(x_t, v, ref, ts, orc.COSINE, 0.1)
+    for b in (0, 2):
+        want = orc.partition(x_t[b:b + 1], v[b:b + 1], ref[b:b + 1], np.float32(ts[b]), orc.COSINE, 0.1)
+        decided = np.abs(want["score"] - np.float32(0.1)) >= 1e-4
+        check_against_oracle({k: a[b:b + 1] for k, a in got.items()}, want, N, decided)
+    assert np.all(got["mask"][1] == 77) and np.all(got["slot"][1] == -7) and got["n_edit"][1] == -7
+    assert np.all(np.isnan(got["score"][1]))
