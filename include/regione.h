@@ -97,6 +97,8 @@ const char* regione_status_string(int status);
  * n_edit      : dev int32 [B]
  * score       : dev f32   [B, N], nullable; receives s
  * Limits: 1 <= N <= 2^20 per request (REGIONE_UNSUPPORTED above), B <= 65535.
+ * One kernel launch per 128 requests; a call of few long requests (N >= 32768, at most 18
+ * requests) takes two per 128, the decisions and then the compaction, with the same results.
  */
 int regione_partition(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
                       int B, int N, int C, const float* t, int metric, float threshold,
@@ -104,12 +106,12 @@ int regione_partition(const regione_bf16* x_t, const regione_bf16* v, const regi
                       int32_t* n_edit, float* score, int32_t* dev_status, void* stream);
 
 /*
- * regione_partition and regione_region_rows (below) in one launch: the partition
+ * regione_partition and regione_region_rows (below) in one call: the partition
  * of Sec. 4 "Adaptive Region Partition" that also writes the joint-sequence row
  * lists of the region-attention layer (Sec. 4 "Region-Aware Generation").  Same
  * arguments, layouts, limits and results as the two calls made one after the
  * other; the row lists are composed while the index lists are written, so the
- * second launch and its pass over the lists are saved.
+ * launch of regione_region_rows and its pass over the lists are saved.
  */
 int regione_partition_rows(const regione_bf16* x_t, const regione_bf16* v, const regione_bf16* ref,
                            int B, int N, int C, const float* t, int metric, float threshold,
