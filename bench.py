@@ -640,7 +640,7 @@ def loop_row(torch, binding, synth, to_dev):
 
 
 def stack_loop_row(torch, binding, synth, to_dev, blocks=8):
-    """Config 4 as BASELINE describes it: the 28-step loop around a stand-in stack of 8 random blocks
+    """The sampler-loop configuration at its stated size: the 28-step loop around a stand-in stack of 8 random blocks
     (hidden 3072, 24 heads x 128, MLP ratio 4; 256 text + 4096 image + 4096 reference tokens), once with
     every step a full step and once under the region-aware schedule (partition after step 6 with the L2
     threshold, cache refreshed every 5 steps, alternate region steps reused).  The blocks' GEMMs,
