@@ -86,7 +86,7 @@ class RegionStep:
         self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=device)
         self.launches = 0
         self._side = torch.cuda.Stream(device=device)
-        self._fork, self._join, self._qkv_ready = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+        self._fork, self._join = torch.cuda.Event(), torch.cuda.Event()
         self.attention_events = None      # optional (start, stop) pair recorded around the attention
 
     def run(self, x_t, v, ref, q_full, k_full, v_full, t, scale, dt, dt_unedited, stream=None,
@@ -101,30 +101,25 @@ class RegionStep:
                          self.keep_idx, self.slot, self.n_edit, s.n_text, s.n_ref, s.membership,
                          self.query_rows, self.n_q, self.cache_rows, self.n_cache, dev_status=st,
                          stream=stream)
-        # Two branches hang off the partition.  The main stream writes the cache (the long HBM pass of the
-        # step) and then runs the attention; the side stream gathers the fresh Q / K / V rows beside the
-        # cache store (both only read the full tensors) and then runs the latent branch (gather of X^E and
-        # v, velocity decay, merge: small latency-bound kernels).  The attention waits for the Q / K / V
-        # gather, the step's end for the latent branch.
+        # Two independent branches hang off the partition: the latent branch (gather of X^E and v,
+        # velocity decay, merge: small latency-bound kernels) and the attention branch (cache store,
+        # gather of Q/K/V, attention, scatter).  The latent branch runs on a side stream so that it
+        # falls into the shadow of the cache store; both join before the step returns.
         main = torch.cuda.current_stream() if stream is None else stream
         self._fork.record(main)
         self._side.wait_event(self._fork)
         side = self._side
-        # (the cache store, the longest wait of the attention, is handed to the driver first; everything on
-        # the side stream fits into its shadow, so nothing competes with the attention for SMs)
-        if store_cache:
-            b.rikv_store(k_full, v_full, self.cache_rows, self.n_cache, self.k_cache, self.v_cache,
-                         dev_status=st, stream=stream)
-        b.gather_multi([q_full, k_full, v_full], self.query_rows, self.n_q,
-                       [self.q_e, self.k_fresh, self.v_fresh], dev_status=st, stream=side)
-        self._qkv_ready.record(side)
         b.gather_multi([x_t, v], self.edit_idx, self.n_edit, [self.x_e, self.v_e], dev_status=st,
                        stream=side)
         b.velocity_decay(self.v_e, scale, dt, self.x_e, self.n_edit, v_cache_out=self.v_avd,
                          dev_status=st, stream=side)
         b.merge(x_t, v, self.x_e, self.slot, dt_unedited, self.x_out, dev_status=st, stream=side)
         self._join.record(side)
-        main.wait_event(self._qkv_ready)
+        if store_cache:
+            b.rikv_store(k_full, v_full, self.cache_rows, self.n_cache, self.k_cache, self.v_cache,
+                         dev_status=st, stream=stream)
+        b.gather_multi([q_full, k_full, v_full], self.query_rows, self.n_q,
+                       [self.q_e, self.k_fresh, self.v_fresh], dev_status=st, stream=stream)
         if self.attention_events is not None:
             self.attention_events[0].record(stream)
         # the attention rows go straight to their positions in the joint sequence (o_full)
